@@ -1,0 +1,389 @@
+"""CPU oracle for the SepLLM attention path (TEST INFRASTRUCTURE, not product code).
+
+A plain, slow, fp64 restatement of what the paper defines, written to be checked
+against the paper by eye.  Only tests, the smoke check and the CPU-baseline leg
+of the benchmark may import it; the CUDA path shares no code with it.
+
+Notation follows the paper: sequence length m is called ``L`` here, ``a`` is
+the number of initial tokens, ``n`` the number of neighbouring tokens, and for
+the streaming cache ``s``, ``w``, ``c`` are the separator-cache, local-window
+and total capacities.
+
+Pins (see tests/test_oracle_*.py): brute-force loops on tiny inputs, the
+dense-causal / sliding-window special cases, row sums, finite differences,
+the closed forms of Eq. 3 and Eq. 4 with the runtime-KV values the paper
+prints, and the attention-map ratio of Table 3.
+
+Parity unpinned (the paper gives no value that separates the alternatives):
+  * the order in which separators leave a full Separator Cache (taken: oldest
+    first), and
+  * whether a streaming step attends before or after compaction (taken:
+    append, compact if full, then attend).
+"""
+from __future__ import annotations
+
+import math
+from typing import Iterable, List, Sequence
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------
+# Mask (Section 3.1; Eq. 2)
+# ----------------------------------------------------------------------------
+
+def separator_flags(token_ids: np.ndarray, sep_ids: Iterable[int]) -> np.ndarray:
+    """f[j] = True iff token j is one of the separator ids (Section 4.1 lists
+    the nine separator strings; here they arrive as ids)."""
+    sep = set(int(x) for x in sep_ids)
+    return np.array([int(t) in sep for t in token_ids], dtype=bool)
+
+
+def mask_matrix(f: np.ndarray, a: int, n: int) -> np.ndarray:
+    """Binary mask M of Eq. 2 for one sequence.
+
+    Query i sees key j (j <= i) iff j is one of the first ``a`` tokens, or j is
+    a separator, or j is among the ``n`` closest tokens, the query's own
+    position counted as the closest (Section 3.1).
+    """
+    L = f.shape[0]
+    i = np.arange(L)[:, None]
+    j = np.arange(L)[None, :]
+    causal = j <= i
+    initial = j < a
+    separator = f[None, :]
+    neighbour = (i - j) < n
+    return causal & (initial | separator | neighbour)
+
+
+def mask_rows(f: np.ndarray, a: int, n: int, rows: np.ndarray) -> np.ndarray:
+    """Rows ``rows`` of the mask of Eq. 2 (same predicate, fewer rows)."""
+    L = f.shape[0]
+    i = np.asarray(rows)[:, None]
+    j = np.arange(L)[None, :]
+    return (j <= i) & ((j < a) | f[None, :] | ((i - j) < n))
+
+
+def kept_pairs(f: np.ndarray, a: int, n: int) -> int:
+    """Number of ones in M, counted row by row from the predicate."""
+    L = f.shape[0]
+    total = 0
+    side = (np.arange(L) < a) | f
+    prefix = np.concatenate([[0], np.cumsum(side)])  # prefix[j] = #side in [0, j)
+    for i in range(L):
+        lo = max(0, i - n + 1)          # first position of the neighbour window
+        total += (i - lo + 1) + int(prefix[lo])
+    return total
+
+
+def attention_map_ratio(f: np.ndarray, a: int, n: int) -> float:
+    """Share of ones in the lower triangle of the mask (Table 3, 'Atten. (%)')."""
+    L = f.shape[0]
+    return kept_pairs(f, a, n) / (L * (L + 1) / 2)
+
+
+# ----------------------------------------------------------------------------
+# Forward (Eq. 1, Eq. 2)
+# ----------------------------------------------------------------------------
+
+def attn_fwd_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, M: np.ndarray,
+                  scale: float | None = None):
+    """Masked softmax attention for one head.
+
+    Q: [R][d] (the R query rows that M's rows describe), K, V: [L][d], M: [R][L].
+    Lambda = Q K^T * scale where M = 1 and -inf elsewhere; A = softmax(Lambda);
+    O = A V.  Returns O [R][d], LSE [R] (natural log), A [R][L].
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    d = Q.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    Lam = (Q @ K.T) * scale
+    Lam = np.where(M, Lam, -np.inf)
+    mx = Lam.max(axis=1, keepdims=True)
+    E = np.exp(Lam - mx)
+    Z = E.sum(axis=1, keepdims=True)
+    A = E / Z
+    O = A @ V
+    LSE = (mx + np.log(Z))[:, 0]
+    return O, LSE, A
+
+
+def attn_fwd(Q: np.ndarray, K: np.ndarray, V: np.ndarray, flags: np.ndarray,
+             a: int, n: int, scale: float | None = None):
+    """Forward for a batch.  Q [B][Hq][L][d], K,V [B][Hkv][L][d], flags [B][L].
+
+    Query head h reads KV head h // (Hq // Hkv).  The mask is the same for all
+    heads (Section 3.2, after Eq. 2).  Returns O [B][Hq][L][d], LSE [B][Hq][L].
+    """
+    B, Hq, L, d = Q.shape
+    G = Hq // K.shape[1]
+    O = np.zeros((B, Hq, L, d))
+    LSE = np.zeros((B, Hq, L))
+    for b in range(B):
+        M = mask_matrix(flags[b], a, n)
+        for h in range(Hq):
+            O[b, h], LSE[b, h], _ = attn_fwd_rows(Q[b, h], K[b, h // G], V[b, h // G], M, scale)
+    return O, LSE
+
+
+# ----------------------------------------------------------------------------
+# Backward (gradient of Eq. 1 under the mask of Eq. 2)
+# ----------------------------------------------------------------------------
+
+def attn_bwd_head(Q, K, V, dO, M, scale: float | None = None):
+    """Gradients of sum(O * dO) for one head, all rows.
+
+    With A = softmax(Lambda): dV = A^T dO; dA = dO V^T;
+    dLambda = A * (dA - rowsum(dA * A)); dQ = dLambda K * scale;
+    dK = dLambda^T Q * scale.  rowsum(dA * A) equals rowsum(dO * O).
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    d = Q.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    O, _, A = attn_fwd_rows(Q, K, V, M, scale)
+    dV = A.T @ dO
+    dA = dO @ V.T
+    delta = (dO * O).sum(axis=1, keepdims=True)
+    dLam = A * (dA - delta)
+    dQ = (dLam @ K) * scale
+    dK = (dLam.T @ Q) * scale
+    return dQ, dK, dV
+
+
+def attn_bwd(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None):
+    """Backward for a batch; dK and dV are summed over the query heads that
+    share a KV head."""
+    B, Hq, L, d = Q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    dQ = np.zeros((B, Hq, L, d))
+    dK = np.zeros((B, Hkv, L, d))
+    dV = np.zeros((B, Hkv, L, d))
+    for b in range(B):
+        M = mask_matrix(flags[b], a, n)
+        for h in range(Hq):
+            q, k, v = attn_bwd_head(Q[b, h], K[b, h // G], V[b, h // G], dO[b, h], M, scale)
+            dQ[b, h] = q
+            dK[b, h // G] += k
+            dV[b, h // G] += v
+    return dQ, dK, dV
+
+
+def attn_rows_fwd_bwd(Q, K, V, dO, f, a: int, n: int, rows, scale: float | None = None):
+    """O, LSE and dQ for selected rows of one head (each is a function of its
+    own row only).  Q, dO: [L][d]; rows: indices.  Used where L is too long to
+    evaluate every row."""
+    rows = np.asarray(rows)
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    d = Q.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    M = mask_rows(f, a, n, rows)
+    O, LSE, A = attn_fwd_rows(Q[rows], K, V, M, scale)
+    dA = dO[rows] @ V.T
+    delta = (dO[rows] * O).sum(axis=1, keepdims=True)
+    dLam = A * (dA - delta)
+    dQ = (dLam @ K) * scale
+    return O, LSE, dQ
+
+
+# ----------------------------------------------------------------------------
+# Index (the data the kernels consume; integers, compared bit for bit)
+# ----------------------------------------------------------------------------
+
+def build_index(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int,
+                side_cap: int):
+    """Canonical index arrays for a batch of sequences.
+
+    side member g[j] = (j < a) or f[j]            (initial tokens and separators)
+    cnt[j]  = number of side members at positions < j, j = 0..L
+    side_pos = ascending positions of side members, n_side = cnt[L]
+    lim[i]  = cnt[max(0, i-n+1)]: side members at distance >= n from query i,
+              i.e. those row i keeps that its neighbour window does not cover
+    tile_meta[t] for the query tile of rows [t*BM, min(L,(t+1)*BM)):
+      0 side_full  = floor(lim[first row] / BN)   side tiles every row sees in full
+      1 side_last  = ceil(lim[last row] / BN)     side tiles some row sees
+      2 win_lo     = max(0, first row - n + 1)    first key of the tile's window
+      3 win_hi     = last row + 1                 one past its last key
+      4 win_tile_lo = win_lo // BN
+      5 win_tile_hi = ceil(win_hi / BN)
+      6 pairs      = kept (query, key) pairs in the tile
+      7 reserved (0)
+    """
+    token_ids = np.asarray(token_ids)
+    B, L = token_ids.shape
+    T = (L + BM - 1) // BM
+    cnt = np.zeros((B, L + 1), dtype=np.int32)
+    lim = np.zeros((B, L), dtype=np.int32)
+    side_pos = np.full((B, side_cap), -1, dtype=np.int32)
+    n_side = np.zeros((B,), dtype=np.int32)
+    tile_meta = np.zeros((B, T, 8), dtype=np.int32)
+    sep = set(int(x) for x in sep_ids)
+    for b in range(B):
+        k = 0
+        for j in range(L):
+            cnt[b, j] = k
+            if j < a or int(token_ids[b, j]) in sep:
+                if k < side_cap:
+                    side_pos[b, k] = j
+                k += 1
+        cnt[b, L] = k
+        n_side[b] = k
+        for i in range(L):
+            lim[b, i] = cnt[b, max(0, i - n + 1)]
+        for t in range(T):
+            r0 = t * BM
+            r1 = min(L, (t + 1) * BM) - 1
+            pairs = 0
+            for i in range(r0, r1 + 1):
+                pairs += int(lim[b, i]) + min(i + 1, n)
+            win_lo = max(0, r0 - n + 1)
+            win_hi = r1 + 1
+            tile_meta[b, t] = [int(lim[b, r0]) // BN, -(-int(lim[b, r1]) // BN), win_lo, win_hi,
+                               win_lo // BN, -(-win_hi // BN), pairs, 0]
+    return dict(cnt=cnt, lim=lim, side_pos=side_pos, n_side=n_side, tile_meta=tile_meta)
+
+
+def build_index_fast(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int,
+                     side_cap: int):
+    """Same arrays as :func:`build_index`, with numpy prefix sums in place of
+    the Python loops, for sequences too long to loop over.  Tests check the two
+    against each other."""
+    token_ids = np.asarray(token_ids)
+    B, L = token_ids.shape
+    T = (L + BM - 1) // BM
+    g = np.isin(token_ids, np.asarray(list(sep_ids))) | (np.arange(L)[None, :] < a)
+    cnt = np.zeros((B, L + 1), dtype=np.int64)
+    cnt[:, 1:] = np.cumsum(g, axis=1)
+    i = np.arange(L)
+    lim = cnt[:, np.maximum(0, i - n + 1)]
+    side_pos = np.full((B, side_cap), -1, dtype=np.int32)
+    for b in range(B):
+        p = np.nonzero(g[b])[0][:side_cap]
+        side_pos[b, :p.size] = p
+    per_row = lim + np.minimum(i + 1, n)[None, :]
+    tile_meta = np.zeros((B, T, 8), dtype=np.int32)
+    for t in range(T):
+        r0 = t * BM
+        r1 = min(L, (t + 1) * BM) - 1
+        win_lo = max(0, r0 - n + 1)
+        win_hi = r1 + 1
+        tile_meta[:, t, 0] = lim[:, r0] // BN
+        tile_meta[:, t, 1] = -(-lim[:, r1] // BN)
+        tile_meta[:, t, 2] = win_lo
+        tile_meta[:, t, 3] = win_hi
+        tile_meta[:, t, 4] = win_lo // BN
+        tile_meta[:, t, 5] = -(-win_hi // BN)
+        tile_meta[:, t, 6] = per_row[:, r0:r1 + 1].sum(axis=1)
+    return dict(cnt=cnt.astype(np.int32), lim=lim.astype(np.int32), side_pos=side_pos,
+                n_side=cnt[:, L].astype(np.int32), tile_meta=tile_meta)
+
+
+# ----------------------------------------------------------------------------
+# Streaming cache (Section 3.3, "Tailored Streaming Design")
+# ----------------------------------------------------------------------------
+
+class StreamingCache:
+    """The four cache blocks as lists of token positions.
+
+    Initial Cache fills first and is never changed.  Every later token enters
+    the neighbour run, whose newest ``w`` entries are the Local Window Cache and
+    whose older entries are the Past Window Cache.  When the runtime size
+    reaches ``c`` the separators of the Past Window Cache move to the Separator
+    Cache in position order and the other Past Window entries are dropped; a
+    Separator Cache holding more than ``s`` entries drops its oldest.
+    """
+
+    def __init__(self, a: int, s: int, w: int, c: int):
+        if not (a + s + w < c):
+            raise ValueError("the paper requires a + s + w < c")
+        self.a, self.s, self.w, self.c = a, s, w, c
+        self.init: List[int] = []
+        self.sep: List[int] = []
+        self.window: List[int] = []      # past window followed by local window
+        self.window_is_sep: List[bool] = []
+        self.next_pos = 0
+        self.compactions = 0
+
+    # sizes in the paper's names
+    @property
+    def size_init(self):
+        return len(self.init)
+
+    @property
+    def size_sep(self):
+        return len(self.sep)
+
+    @property
+    def size_local_w(self):
+        return min(len(self.window), self.w)
+
+    @property
+    def size_past_w(self):
+        return len(self.window) - self.size_local_w
+
+    @property
+    def n(self):
+        return len(self.window)
+
+    @property
+    def size_run(self):
+        return len(self.init) + len(self.sep) + len(self.window)
+
+    def update(self, is_sep: bool) -> None:
+        """Take in the next token of the stream."""
+        pos = self.next_pos
+        self.next_pos += 1
+        if len(self.init) < self.a:
+            self.init.append(pos)
+            return
+        self.window.append(pos)
+        self.window_is_sep.append(bool(is_sep))
+        if self.size_run == self.c:
+            n_past = len(self.window) - self.w
+            moved = [p for p, f in zip(self.window[:n_past], self.window_is_sep[:n_past]) if f]
+            self.sep.extend(moved)
+            if len(self.sep) > self.s:
+                self.sep = self.sep[len(self.sep) - self.s:]
+            self.window = self.window[n_past:]
+            self.window_is_sep = self.window_is_sep[n_past:]
+            self.compactions += 1
+
+    def retained(self) -> List[int]:
+        """Positions whose K/V the next decode step attends to."""
+        return self.init + self.sep + self.window
+
+
+def avg_neighbour_limit(w: int, c: int, a: int, s: int) -> float:
+    """Eq. 3: long-run mean of n."""
+    return (w + c - a - s) / 2.0
+
+
+def avg_runtime_kv_limit(w: int, c: int, a: int, s: int) -> float:
+    """Eq. 4: long-run mean of Size_run."""
+    return (w + c + a + s) / 2.0
+
+
+def decode_attention(q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, scale: float | None = None):
+    """One query over a retained set: q [d], Kc, Vc [R][d].  Returns o [d], lse."""
+    q = np.asarray(q, dtype=np.float64)
+    Kc = np.asarray(Kc, dtype=np.float64)
+    Vc = np.asarray(Vc, dtype=np.float64)
+    d = q.shape[0]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    lam = (Kc @ q) * scale
+    mx = lam.max()
+    e = np.exp(lam - mx)
+    Z = e.sum()
+    return (e / Z) @ Vc, mx + math.log(Z)

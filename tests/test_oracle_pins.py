@@ -1,0 +1,294 @@
+"""Pins that hold the CPU oracle to the paper and to textbook routines.
+
+None of these retype the oracle's own formula: they use Python-loop brute
+force built from the paper's wording, torch's dense attention and autograd,
+closed forms and values the paper prints.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sepllm_oracle as orc
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_case(seed, L, d, p):
+    g = np.random.default_rng(seed)
+    f = g.random(L) < p
+    Q = g.standard_normal((L, d))
+    K = g.standard_normal((L, d))
+    V = g.standard_normal((L, d))
+    dO = g.standard_normal((L, d))
+    return f, Q, K, V, dO
+
+
+def _kept_set_from_words(f, a, n, i):
+    """Section 3.1 in words: the first a tokens, every separator before the
+    current token, the n closest tokens (the current one included)."""
+    kept = set(range(min(a, i + 1)))
+    kept |= {j for j in range(i + 1) if f[j]}
+    kept |= {j for j in range(i, max(-1, i - n), -1)}
+    return kept
+
+
+@pytest.mark.parametrize("a,n", [(0, 1), (0, 3), (2, 1), (3, 5), (4, 64), (1, 200)])
+def test_mask_matches_set_construction(a, n):
+    f, *_ = _rand_case(a * 100 + n, 96, 4, 0.15)
+    M = orc.mask_matrix(f, a, n)
+    for i in range(96):
+        assert set(np.nonzero(M[i])[0].tolist()) == _kept_set_from_words(f, a, n, i)
+    rows = np.array([0, 5, 50, 95])
+    assert (orc.mask_rows(f, a, n, rows) == M[rows]).all()
+
+
+@pytest.mark.parametrize("a,n", [(0, 1), (2, 4), (4, 16)])
+def test_forward_matches_python_loops(a, n):
+    L, d = 40, 8
+    f, Q, K, V, _ = _rand_case(7 + a + n, L, d, 0.2)
+    O, LSE, A = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(f, a, n))
+    for i in range(L):
+        kept = sorted(_kept_set_from_words(f, a, n, i))
+        lam = [sum(Q[i][t] * K[j][t] for t in range(d)) / math.sqrt(d) for j in kept]
+        mx = max(lam)
+        e = [math.exp(x - mx) for x in lam]
+        Z = sum(e)
+        o = [sum(e[k] / Z * V[j][t] for k, j in enumerate(kept)) for t in range(d)]
+        assert np.allclose(O[i], o, rtol=1e-12, atol=1e-13)
+        assert abs(LSE[i] - (mx + math.log(Z))) < 1e-12
+        assert abs(A[i].sum() - 1.0) < 1e-12
+        assert all(A[i][j] == 0.0 for j in range(L) if j not in kept)
+
+
+def _torch_dense(Q, K, V, mask=None, causal=False):
+    q, k, v = (torch.from_numpy(x)[None, None] for x in (Q, K, V))
+    m = None if mask is None else torch.from_numpy(mask)[None, None]
+    return torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=m, is_causal=causal)[0, 0].numpy()
+
+
+def test_dense_causal_special_cases():
+    L, d = 128, 16
+    f, Q, K, V, _ = _rand_case(3, L, d, 0.1)
+    ref = _torch_dense(Q, K, V, causal=True)
+    # n >= L: every earlier token is a neighbour
+    O1, _, _ = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(f, 2, L))
+    # every token a separator
+    O2, _, _ = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(np.ones(L, bool), 0, 1))
+    assert np.allclose(O1, ref, atol=1e-12)
+    assert np.allclose(O2, ref, atol=1e-12)
+
+
+def test_sliding_window_and_streaming_special_cases():
+    L, d, n = 96, 8, 7
+    _, Q, K, V, _ = _rand_case(5, L, d, 0.0)
+    none = np.zeros(L, bool)
+    band = torch.ones(L, L, dtype=torch.bool).tril().triu(-(n - 1)).numpy()
+    O, _, _ = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(none, 0, n))
+    assert np.allclose(O, _torch_dense(Q, K, V, mask=band), atol=1e-12)
+    # initial + neighbouring tokens only (the StreamingLLM mask)
+    a = 3
+    sink = band.copy()
+    sink[:, :a] = True
+    sink &= np.tril(np.ones((L, L), bool))
+    O, _, _ = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(none, a, n))
+    assert np.allclose(O, _torch_dense(Q, K, V, mask=sink), atol=1e-12)
+
+
+def test_backward_matches_autograd_and_gqa_sum():
+    B, Hq, Hkv, L, d, a, n = 2, 4, 2, 48, 8, 2, 5
+    g = np.random.default_rng(11)
+    flags = g.random((B, L)) < 0.2
+    Q = g.standard_normal((B, Hq, L, d))
+    K = g.standard_normal((B, Hkv, L, d))
+    V = g.standard_normal((B, Hkv, L, d))
+    dO = g.standard_normal((B, Hq, L, d))
+    dQ, dK, dV = orc.attn_bwd(Q, K, V, dO, flags, a, n)
+    O, LSE = orc.attn_fwd(Q, K, V, flags, a, n)
+    q, k, v = (torch.tensor(x, requires_grad=True) for x in (Q, K, V))
+    G = Hq // Hkv
+    kk = k.repeat_interleave(G, dim=1)
+    vv = v.repeat_interleave(G, dim=1)
+    M = torch.stack([torch.from_numpy(orc.mask_matrix(flags[b], a, n)) for b in range(B)])[:, None]
+    lam = (q @ kk.transpose(-1, -2)) / math.sqrt(d)
+    lam = lam.masked_fill(~M, float("-inf"))
+    o = torch.softmax(lam, dim=-1) @ vv
+    (o * torch.tensor(dO)).sum().backward()
+    assert np.allclose(O, o.detach().numpy(), atol=1e-12)
+    assert np.allclose(LSE, torch.logsumexp(lam, dim=-1).detach().numpy(), atol=1e-12)
+    assert np.allclose(dQ, q.grad.numpy(), atol=1e-11)
+    assert np.allclose(dK, k.grad.numpy(), atol=1e-11)
+    assert np.allclose(dV, v.grad.numpy(), atol=1e-11)
+
+
+def test_backward_matches_finite_differences():
+    L, d, a, n = 24, 4, 1, 3
+    f, Q, K, V, dO = _rand_case(21, L, d, 0.25)
+    M = orc.mask_matrix(f, a, n)
+    dQ, dK, dV = orc.attn_bwd_head(Q, K, V, dO, M)
+
+    def loss(q, k, v):
+        return float((orc.attn_fwd_rows(q, k, v, M)[0] * dO).sum())
+
+    h = 1e-6
+    g = np.random.default_rng(0)
+    for X, dX, which in ((Q, dQ, 0), (K, dK, 1), (V, dV, 2)):
+        for _ in range(12):
+            i, t = int(g.integers(L)), int(g.integers(d))
+            Xp, Xm = X.copy(), X.copy()
+            Xp[i, t] += h
+            Xm[i, t] -= h
+            args_p = [Q, K, V]
+            args_m = [Q, K, V]
+            args_p[which] = Xp
+            args_m[which] = Xm
+            fd = (loss(*args_p) - loss(*args_m)) / (2 * h)
+            assert abs(fd - dX[i, t]) <= 1e-6 * max(1.0, abs(fd))
+
+
+def test_rows_variant_matches_full():
+    L, d, a, n = 80, 8, 2, 6
+    f, Q, K, V, dO = _rand_case(33, L, d, 0.2)
+    M = orc.mask_matrix(f, a, n)
+    O, LSE, _ = orc.attn_fwd_rows(Q, K, V, M)
+    dQ, _, _ = orc.attn_bwd_head(Q, K, V, dO, M)
+    rows = np.array([0, 1, 17, 79])
+    o, lse, dq = orc.attn_rows_fwd_bwd(Q, K, V, dO, f, a, n, rows)
+    assert np.allclose(o, O[rows]) and np.allclose(lse, LSE[rows]) and np.allclose(dq, dQ[rows])
+
+
+# ---------------------------------------------------------------- Table 3
+def test_attention_map_ratio_table3():
+    for line in open(os.path.join(GOLD, "attention_map_ratio.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        L, a, n, printed = line.split()
+        r = 100.0 * orc.attention_map_ratio(np.zeros(int(L), bool), int(a), int(n))
+        assert f"{r:.2f}" == printed
+    # brute-force count equals the row-wise count
+    f, *_ = _rand_case(2, 200, 2, 0.12)
+    assert orc.kept_pairs(f, 4, 16) == int(orc.mask_matrix(f, 4, 16).sum())
+
+
+# ---------------------------------------------------------------- Eq. 3 / Eq. 4
+def _golden_rkv():
+    rows = []
+    for line in open(os.path.join(GOLD, "runtime_kv_table.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        a, s, w, c, r = (int(x) for x in line.split()[:5])
+        rows.append((a, s, w, c, r))
+    return rows
+
+
+def test_eq4_reproduces_printed_runtime_kv():
+    rows = _golden_rkv()
+    assert len(rows) == 10
+    for a, s, w, c, printed in rows:
+        assert orc.avg_runtime_kv_limit(w, c, a, s) == printed
+        assert orc.avg_neighbour_limit(w, c, a, s) + a + s == printed
+
+
+@pytest.mark.parametrize("a,s,w,c,printed", _golden_rkv()[:4] + _golden_rkv()[6:7])
+def test_streaming_cache_simulation_meets_eq3_eq4(a, s, w, c, printed):
+    g = np.random.default_rng(c + s)
+    cache = orc.StreamingCache(a, s, w, c)
+    period = c - a - s - w
+    T = 60 * period + 4 * c
+    sizes, ns = [], []
+    first_full = None
+    for t in range(T):
+        cache.update(bool(g.random() < 0.3))
+        assert cache.size_run <= c
+        assert cache.size_run == cache.size_init + cache.size_sep + cache.size_past_w + cache.size_local_w
+        assert cache.size_local_w <= w and cache.size_sep <= s and cache.size_init <= a
+        if first_full is None and cache.size_sep == s and cache.compactions > 0:
+            first_full = t
+        if first_full is not None and t >= first_full + period:
+            sizes.append(cache.size_run)
+            ns.append(cache.n)
+            assert w <= cache.n <= c - a - s
+    assert min(ns) == w
+    k = (len(ns) // period) * period      # whole periods
+    assert abs(np.mean(sizes[:k]) - printed) <= 0.5
+    assert abs(np.mean(ns[:k]) - orc.avg_neighbour_limit(w, c, a, s)) <= 0.5
+
+
+def test_streaming_cache_keeps_what_the_mask_keeps():
+    """With room for every separator, the retained set at step t is row t of
+    the mask with n = the current length of the neighbour run."""
+    a, s, w = 3, 100, 8
+    g = np.random.default_rng(4)
+    f = g.random(600) < 0.2
+    cache = orc.StreamingCache(a, s, w, a + s + w + 13)
+    checked_after_compaction = 0
+    for t in range(600):
+        cache.update(bool(f[t]))
+        if cache.size_sep < s:        # nothing evicted yet
+            row = orc.mask_rows(f, a, cache.n, np.array([t]))[0]
+            assert sorted(cache.retained()) == np.nonzero(row)[0].tolist()
+            checked_after_compaction += cache.compactions > 0
+    assert cache.compactions >= 3 and checked_after_compaction > 50
+
+
+def test_streaming_cache_fifo_and_order():
+    cache = orc.StreamingCache(1, 2, 2, 8)
+    flags = [0, 1, 1, 0, 1, 1, 1, 1, 0, 0, 1, 0, 0, 0]
+    for fl in flags:
+        cache.update(bool(fl))
+    # step by step by hand: init=[0]; window fills 1..7 -> size 8 == c at pos 7:
+    # past = [1..5], separators there 1,2,4,5 -> sep keeps the newest two [4,5]
+    # window = [6,7]; then 8,9,10 appended (size 1+2+5 = 8 at pos 10):
+    # past = [6,7,8], separators 6,7 -> sep = [6,7]; window = [9,10]; then 11,12,13
+    # size = 1+2+5 = 8 at pos 13: past = [9,10,11], separator 10 -> sep = [7,10]
+    assert cache.init == [0]
+    assert cache.sep == [7, 10]
+    assert cache.window == [12, 13]
+
+
+# ---------------------------------------------------------------- decode
+def test_decode_equals_last_prefill_row():
+    L, d, a, n = 70, 8, 2, 9
+    f, Q, K, V, _ = _rand_case(9, L, d, 0.2)
+    O, LSE, _ = orc.attn_fwd_rows(Q, K, V, orc.mask_matrix(f, a, n))
+    t = L - 1
+    kept = sorted(_kept_set_from_words(f, a, n, t))
+    o, lse = orc.decode_attention(Q[t], K[kept], V[kept])
+    assert np.allclose(o, O[t], atol=1e-13) and abs(lse - LSE[t]) < 1e-12
+    o1, lse1 = orc.decode_attention(Q[t], K[5:6], V[5:6])
+    assert np.allclose(o1, V[5])
+
+
+# ---------------------------------------------------------------- index
+@pytest.mark.parametrize("L,a,n,BM,BN", [(300, 4, 64, 128, 128), (129, 0, 1, 128, 128), (64, 3, 500, 32, 16)])
+def test_index_invariants(L, a, n, BM, BN):
+    g = np.random.default_rng(L)
+    sep_ids = [5, 7, 9]
+    ids = g.integers(0, 40, size=(2, L)).astype(np.int32)
+    idx = orc.build_index(ids, sep_ids, a, n, BM, BN, side_cap=L)
+    fast = orc.build_index_fast(ids, sep_ids, a, n, BM, BN, side_cap=L)
+    for k in idx:
+        assert idx[k].dtype == fast[k].dtype and (idx[k] == fast[k]).all(), k
+    for b in range(2):
+        f = orc.separator_flags(ids[b], sep_ids)
+        M = orc.mask_matrix(f, a, n)
+        cnt, lim, sp, ns = idx["cnt"][b], idx["lim"][b], idx["side_pos"][b], int(idx["n_side"][b])
+        assert (np.diff(cnt) >= 0).all() and cnt[L] == ns
+        assert (np.diff(sp[:ns]) > 0).all() and (sp[ns:] == -1).all()
+        assert (np.diff(lim) >= 0).all() and (lim <= cnt[1:]).all()
+        # row i keeps exactly side entries [0, lim[i]) plus its window
+        for i in range(L):
+            kept = set(sp[:lim[i]].tolist()) | set(range(max(0, i - n + 1), i + 1))
+            assert kept == set(np.nonzero(M[i])[0].tolist())
+            assert len(kept) == lim[i] + min(i + 1, n)      # the two parts are disjoint
+        assert idx["tile_meta"][b, :, 6].sum() == M.sum() == orc.kept_pairs(f, a, n)
+        T = (L + BM - 1) // BM
+        for t in range(T):
+            sf, sl, wl, wh, tl, th, _, z = idx["tile_meta"][b, t]
+            rows = range(t * BM, min(L, (t + 1) * BM))
+            assert sf * BN <= min(lim[i] for i in rows) < (sf + 1) * BN
+            assert (sl - 1) * BN < max(lim[i] for i in rows) <= sl * BN or (sl == 0 and max(lim[i] for i in rows) == 0)
+            assert wl == max(0, rows[0] - n + 1) and wh == rows[-1] + 1
+            assert tl * BN <= wl < (tl + 1) * BN and (th - 1) * BN < wh <= th * BN and z == 0

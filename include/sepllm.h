@@ -1,0 +1,207 @@
+/*
+ * libsepllm — separator-masked causal attention for one B200 (sm_100a).
+ *
+ * The operations follow "SepLLM" (arXiv 2412.12094): a query at position i
+ * attends to the first n_init tokens, to every earlier separator token and to
+ * its n_neighbor closest tokens, itself included (Section 3.1; Eq. 1 and
+ * Eq. 2), in forward and backward; generation keeps a four-block KV cache
+ * (Section 3.3).
+ *
+ * Conventions for every call
+ *  - C ABI, plain pointers and sizes.  "dev" = device pointer, "host" = host
+ *    pointer.  Descriptors are host structs read during the call.
+ *  - The caller owns every buffer.  Unless a call says otherwise the library
+ *    allocates nothing and keeps no state between calls.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *    only enqueue work; they do not synchronise unless stated.
+ *  - Errors are return codes.  Shape, alignment and capacity errors are found
+ *    on the host before anything is launched.  Conditions only the device can
+ *    see (more side entries than side_cap, a wait that ran out) are written to
+ *    a status word at the start of the workspace / state buffer and read with
+ *    sepllm_last_device_status(); kernels clamp instead of writing out of
+ *    bounds.
+ *  - Tensors are bf16 (two bytes, upper half of an IEEE fp32), row-major,
+ *    contiguous, base pointers 16-byte aligned:
+ *        Q, O, dO, dQ : [B][Hq][L][d]        K, V, dK, dV : [B][Hkv][L][d]
+ *        LSE          : [B][Hq][L] fp32, natural logarithm
+ *    Query head h reads KV head h / (Hq/Hkv).
+ *  - Supported: d in {64, 128}; Hq a multiple of Hkv; n_neighbor >= 1;
+ *    n_init >= 0; index tiles BM = BN = 128 for the attention calls.
+ */
+#ifndef SEPLLM_H_
+#define SEPLLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int sepllm_status;
+enum {
+  SEPLLM_OK = 0,
+  SEPLLM_INVALID_ARG = 1,       /* null pointer, non-positive size, misaligned buffer */
+  SEPLLM_UNSUPPORTED = 2,       /* valid request outside the supported set above */
+  SEPLLM_BUFFER_TOO_SMALL = 3,
+  SEPLLM_CUDA_ERROR = 4,        /* a CUDA runtime / driver call failed */
+  SEPLLM_CAPACITY_EXCEEDED = 5, /* device status: more side entries than side_cap */
+  SEPLLM_TIMEOUT = 6,           /* device status: a bounded wait in a kernel ran out */
+  SEPLLM_NOT_BUILT = 7
+};
+
+#define SEPLLM_MAX_SEP_IDS 64
+
+/* Index description.  side_cap = capacity (entries per sequence) of the side
+ * list, i.e. initial tokens plus separators; L is always enough. */
+typedef struct {
+  int32_t B, L, n_init, n_neighbor, n_sep, BM, BN, side_cap;
+} sepllm_index_desc;
+
+/* scale = 0 means 1/sqrt(d) (Eq. 1).  grad_dtype: 0 = bf16, 1 = fp32 outputs
+ * for dQ, dK, dV. */
+typedef struct {
+  int32_t B, Hq, Hkv, d, L;
+  float scale;
+  int32_t grad_dtype;
+} sepllm_attn_desc;
+
+/* Streaming cache capacities in the paper's names (Section 3.3): a initial,
+ * s separator, w local window, c total; a + s + w < c, w >= 1. */
+typedef struct {
+  int32_t B, Hkv, Hq, d, a, s, w, c;
+} sepllm_cache_desc;
+
+/* ---- index blob -----------------------------------------------------------
+ * The index is one device buffer: this header, then five int32 arrays at the
+ * byte offsets it gives (each 256-byte aligned):
+ *   cnt       [B][L+1]      cnt[j] = side members (j < n_init or separator) at positions < j
+ *   lim       [B][L]        lim[i] = cnt[max(0, i-n_neighbor+1)]: side entries row i keeps
+ *                           outside its neighbour window
+ *   side_pos  [B][side_cap] ascending positions of side members (-1 beyond n_side)
+ *   n_side    [B]           number of side members (may exceed side_cap: then the status
+ *                           word reads SEPLLM_CAPACITY_EXCEEDED and side_pos is truncated)
+ *   tile_meta [B][ceil(L/BM)][8] per query tile of BM rows:
+ *       0 side_full   floor(lim[first row]/BN)   side tiles all rows see in full
+ *       1 side_last   ceil(lim[last row]/BN)     side tiles any row sees
+ *       2 win_lo      max(0, first row - n_neighbor + 1)
+ *       3 win_hi      last row + 1
+ *       4 win_tile_lo win_lo / BN
+ *       5 win_tile_hi ceil(win_hi / BN)
+ *       6 pairs       kept (query,key) pairs in the tile
+ *       7 0
+ * The mask these arrays encode is Eq. 2 with M[i][j] = 1 iff j <= i and
+ * (j < n_init or token j is a separator or i - j < n_neighbor).
+ */
+#define SEPLLM_INDEX_MAGIC 0x58444953u /* "SIDX" */
+typedef struct {
+  int32_t status;      /* device status word of sepllm_build_index (first word) */
+  uint32_t magic, version;
+  sepllm_index_desc desc;
+  int32_t n_tiles;     /* ceil(L/BM) */
+  int64_t off_cnt, off_lim, off_side_pos, off_n_side, off_tile_meta, total_bytes;
+  int64_t reserved[20];
+} sepllm_index_header; /* 256 bytes */
+
+/* Sizes of the index blob and of the scratch buffer sepllm_build_index needs. */
+sepllm_status sepllm_index_bytes(const sepllm_index_desc* desc, size_t* index_bytes,
+                                 size_t* scratch_bytes);
+
+/* Builds the index of Eq. 2's mask from token ids (Section 3.1: initial,
+ * separator and neighbouring tokens; Section 4.1 for the separator set).
+ *   token_ids dev  int32 [B][L]
+ *   sep_ids   host int32 [n_sep], n_sep <= SEPLLM_MAX_SEP_IDS (0 = no separators)
+ *   index     dev  sepllm_index_bytes() bytes, 256-byte aligned; written in full
+ *   scratch   dev  scratch_bytes, 256-byte aligned; contents undefined afterwards
+ * Integer output, deterministic. */
+sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* token_ids,
+                                 const int32_t* sep_ids, void* index, void* scratch,
+                                 void* stream);
+
+/* Workspace sizes for the attention calls (bytes; either pointer may be NULL). */
+sepllm_status sepllm_attn_workspace_bytes(const sepllm_attn_desc* desc,
+                                          const sepllm_index_desc* idesc, size_t* fwd_bytes,
+                                          size_t* bwd_bytes);
+
+/* Forward of Eq. 1 under the mask of Eq. 2: O = softmax(Q K^T * scale | M) V and
+ * the row log-sum-exp.  Q, K, V dev bf16; index dev (built with the same B, L and
+ * BM = BN = 128); O dev bf16; LSE dev fp32; workspace dev fwd_bytes, 256-byte
+ * aligned (its first word is the device status). */
+sepllm_status sepllm_attn_fwd(const sepllm_attn_desc* desc, const sepllm_index_desc* idesc,
+                              const void* Q, const void* K, const void* V, const void* index,
+                              void* O, float* LSE, void* workspace, void* stream);
+
+/* Backward of the same operation (the gradient of softmax attention, training
+ * with the mask: Section 3.1 "Separator Tokens", Section 4.3): given dO, the
+ * inputs and the forward's O and LSE, writes dQ [B][Hq][L][d] and dK, dV
+ * [B][Hkv][L][d] (summed over the query heads sharing a KV head) in
+ * desc->grad_dtype.  Deterministic: no floating-point atomics.  workspace dev
+ * bwd_bytes, 256-byte aligned. */
+sepllm_status sepllm_attn_bwd(const sepllm_attn_desc* desc, const sepllm_index_desc* idesc,
+                              const void* dO, const void* Q, const void* K, const void* V,
+                              const void* O, const float* LSE, const void* index, void* dQ,
+                              void* dK, void* dV, void* workspace, void* stream);
+
+/* ---- streaming cache (Section 3.3, Tailored Streaming Design) --------------
+ * Kc and Vc are bf16 [B][Hkv][slots][d] with slots = c + s: slots [0,a) are the
+ * Initial Cache, [a, a+s) a ring holding the Separator Cache, [a+s, c+s) a ring
+ * holding the neighbour run whose newest w entries are the Local Window Cache
+ * and whose older entries are the Past Window Cache.  `state` holds the sizes,
+ * ring starts, per-slot token position (int64) and separator flag of every
+ * sequence; its first word is the device status.  Saving and restoring a cache
+ * is a copy of state, Kc and Vc.
+ */
+#define SEPLLM_CACHE_MAGIC 0x48434353u /* "SCCH" */
+typedef struct {
+  int32_t status;                /* device status word (first word) */
+  uint32_t magic, version;
+  int32_t slots;                 /* c + s */
+  sepllm_cache_desc desc;
+  int64_t off_seq, off_slot_pos, off_slot_is_sep, total_bytes;
+  int64_t reserved[22];
+} sepllm_cache_header; /* 256 bytes */
+
+/* Per-sequence record inside the state, 16 int32. */
+typedef struct {
+  int32_t size_init, sep_start, size_sep, win_start, size_win, compactions;
+  int64_t next_pos;              /* tokens seen so far */
+  int32_t reserved[8];
+} sepllm_cache_seq;
+
+/* state_bytes: the state buffer; kv_bytes: ONE of Kc / Vc. */
+sepllm_status sepllm_cache_bytes(const sepllm_cache_desc* desc, size_t* state_bytes,
+                                 size_t* kv_bytes);
+
+/* Empties the cache (writes the whole state buffer). */
+sepllm_status sepllm_cache_init(const sepllm_cache_desc* desc, void* state, void* stream);
+
+/* Takes in one token per sequence: fills the Initial Cache first, then appends
+ * to the neighbour run; when Size_run reaches c the separators of the Past
+ * Window Cache move, in position order, to the Separator Cache, which drops its
+ * oldest entries beyond s, and the other Past Window entries are dropped.
+ *   new_token_ids dev int32 [B]; sep_ids host int32 [n_sep];
+ *   k_new, v_new dev bf16 [B][Hkv][d]. */
+sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, void* Kc, void* Vc,
+                                  const int32_t* new_token_ids, const int32_t* sep_ids,
+                                  int32_t n_sep, const void* k_new, const void* v_new,
+                                  void* stream);
+
+sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* desc, size_t* bytes);
+
+/* One query per sequence over every retained entry (Section 3.2 "Generation",
+ * Section 3.3): o = softmax(q Kc^T * scale) Vc.  q dev bf16 [B][Hq][d]; o dev bf16
+ * [B][Hq][d]; lse dev fp32 [B][Hq] (may be NULL); scale 0 = 1/sqrt(d). */
+sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const void* q,
+                            const void* state, const void* Kc, const void* Vc, void* o,
+                            float* lse, void* workspace, void* stream);
+
+/* Copies the device status word at the start of an index, workspace or state
+ * buffer to *out (host) after synchronising `stream`. */
+sepllm_status sepllm_last_device_status(const void* buffer, int32_t* out, void* stream);
+
+const char* sepllm_status_string(sepllm_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEPLLM_H_ */

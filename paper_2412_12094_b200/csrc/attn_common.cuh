@@ -1,0 +1,35 @@
+// Declarations shared by the attention translation units.
+#pragma once
+#include "common.cuh"
+
+namespace sepllm {
+
+constexpr int kBM = 128, kBN = 128;
+constexpr uint32_t kTileBlockBytes = 128 * 128;  // 128 rows x 64 bf16, one swizzled block
+
+struct AttnLayout {
+  int cap_pad;  // side_cap rounded up to 128 rows
+  // forward workspace: status | Kside | Vside
+  size_t off_ks, off_vs, fwd_bytes;
+  // backward workspace: status | Kside | Vside | Delta | dKside | dVside
+  size_t off_delta, off_dks, off_dvs, bwd_bytes;
+};
+
+sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id);
+AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id);
+sepllm_status fill_index_header(const sepllm_index_desc* d, sepllm_index_header* h);
+
+template <int D>
+__global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
+                               const __nv_bfloat16* __restrict__ V,
+                               const int32_t* __restrict__ side_pos,
+                               const int32_t* __restrict__ n_side, int L, int Hkv, int side_cap,
+                               int cap_pad, __nv_bfloat16* __restrict__ Ks,
+                               __nv_bfloat16* __restrict__ Vs);
+
+// Launches the gather of K/V rows at the side positions into Ks / Vs ([B][Hkv][cap_pad][d]).
+void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
+                   const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
+                   void* Ks, void* Vs, cudaStream_t stream);
+
+}  // namespace sepllm

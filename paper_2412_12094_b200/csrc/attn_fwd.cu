@@ -1,0 +1,494 @@
+// Forward of separator-masked attention (Eq. 1 under the mask of Eq. 2) for sm_100a.
+//
+// Per query tile of 128 rows the kept keys fall in two groups that never overlap:
+//   side   entries [0, lim[i]) of the per-sequence side buffer (initial tokens and separators at
+//          distance >= n from the row), gathered once into contiguous K/V side buffers;
+//   window keys i-n < j <= i, read from K/V in place.
+// One CTA walks the side tiles and then the window tiles of its query tile: TMA brings 128-key
+// K/V tiles into shared memory, tcgen05 MMAs compute S = Q K^T into tensor memory, the CTA's 128
+// threads (one per query row, matching tensor-memory lanes) run the online softmax, P goes back
+// through shared memory as bf16 and a second MMA accumulates O += P V in tensor memory.  Only
+// tiles crossing lim[], the diagonal or the window's left edge are masked element by element.
+#include "attn_common.cuh"
+
+namespace sepllm {
+
+// ---------------------------------------------------------------------------
+// host: tensor maps
+// ---------------------------------------------------------------------------
+EncodeTiledFn get_encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) !=
+          cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+sepllm_status make_tile_map(CUtensorMap* map, const void* base, int d, int64_t rows,
+                            int64_t planes, int64_t row_stride_elems, int64_t plane_stride_elems,
+                            int box_rows) {
+  EncodeTiledFn enc = get_encode_tiled();
+  if (!enc) return SEPLLM_CUDA_ERROR;
+  if (!aligned(base, 16) || (row_stride_elems * 2) % 16 != 0 || (plane_stride_elems * 2) % 16 != 0)
+    return SEPLLM_INVALID_ARG;
+  cuuint64_t dims[3] = {cuuint64_t(d), cuuint64_t(rows), cuuint64_t(planes)};
+  cuuint64_t strides[2] = {cuuint64_t(row_stride_elems) * 2, cuuint64_t(plane_stride_elems) * 2};
+  cuuint32_t box[3] = {64, cuuint32_t(box_rows), 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
+                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SEPLLM_OK : SEPLLM_CUDA_ERROR;
+}
+
+// ---------------------------------------------------------------------------
+// side K/V gather
+// ---------------------------------------------------------------------------
+// grid (ceil(cap_pad / rows_per_block), Hkv, B).  Row r of the side buffer is K/V row
+// side_pos[r]; rows from n_side up to the next multiple of 128 are zero so that the tile holding
+// the last entries contains only finite numbers.
+template <int D>
+__global__ void __launch_bounds__(256)
+gather_side_kv(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+               const int32_t* __restrict__ side_pos, const int32_t* __restrict__ n_side, int L,
+               int Hkv, int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
+               __nv_bfloat16* __restrict__ Vs) {
+  constexpr int LPR = D / 8;
+  constexpr int RPB = 256 / LPR;
+  const int b = blockIdx.z, hk = blockIdx.y;
+  const int r = blockIdx.x * RPB + threadIdx.x / LPR, l = threadIdx.x % LPR;
+  const int ns = min(n_side[b], side_cap);
+  const int ns_pad = min(cap_pad, (ns + 127) / 128 * 128);
+  if (r >= ns_pad) return;
+  const size_t plane = size_t(b) * Hkv + hk;
+  uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+  if (r < ns) {
+    const int pos = side_pos[size_t(b) * side_cap + r];
+    if (pos >= 0 && pos < L) {
+      kv = *reinterpret_cast<const uint4*>(K + (plane * L + pos) * D + l * 8);
+      vv = *reinterpret_cast<const uint4*>(V + (plane * L + pos) * D + l * 8);
+    }
+  }
+  *reinterpret_cast<uint4*>(Ks + (plane * cap_pad + r) * D + l * 8) = kv;
+  *reinterpret_cast<uint4*>(Vs + (plane * cap_pad + r) * D + l * 8) = vv;
+}
+
+// ---------------------------------------------------------------------------
+// forward kernel
+// ---------------------------------------------------------------------------
+template <int D>
+struct FwdSmem {
+  static constexpr int NB = D / 64;  // 64-column blocks per row
+  static constexpr uint32_t kQ = 0;
+  static constexpr uint32_t kK = kQ + NB * kTileBlockBytes;
+  static constexpr uint32_t kV = kK + 2 * NB * kTileBlockBytes;
+  static constexpr uint32_t kP = kV + 2 * NB * kTileBlockBytes;
+  static constexpr uint32_t kBar = kP + 2 * kTileBlockBytes;
+  static constexpr uint32_t kTotal = kBar + 256;
+  // one CTA per SM: each CTA takes all 512 tensor-memory columns
+  static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
+};
+
+struct FwdParams {
+  const int32_t* lim;        // [B][L]
+  const int32_t* tile_meta;  // [B][T][8]
+  __nv_bfloat16* O;
+  float* LSE;
+  int32_t* status;
+  int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap;
+  float scale_log2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKs,
+                const __grid_constant__ CUtensorMap mapVs, const FwdParams p) {
+  using SM = FwdSmem<D>;
+  constexpr int NB = SM::NB;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~uintptr_t(1023));
+  uint8_t* sQ = smem + SM::kQ;
+  uint8_t* sK = smem + SM::kK;
+  uint8_t* sV = smem + SM::kV;
+  uint8_t* sP = smem + SM::kP;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBar);
+  uint64_t* bar_q = bars + 0;
+  uint64_t* bar_k = bars + 1;  // [2]
+  uint64_t* bar_v = bars + 3;  // [2]
+  uint64_t* bar_s = bars + 5;  // [2]
+  uint64_t* bar_o = bars + 7;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const bool leader = (tid == 0);
+  const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
+  const int hq = blockIdx.y, b = blockIdx.z;
+  const int G = p.Hq / p.Hkv;
+  const int q_plane = b * p.Hq + hq;
+  const int kv_plane = b * p.Hkv + hq / G;
+
+  if (leader) {
+    mbar_init(bar_q, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_k + i, 1); mbar_init(bar_v + i, 1); mbar_init(bar_s + i, 1); }
+    mbar_init(bar_o, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
+    tma_prefetch_desc(&mapKs); tma_prefetch_desc(&mapVs);
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_row = tmem + (uint32_t(warp * 32) << 16);
+  const uint32_t tmem_S0 = 0, tmem_O = 256;
+
+  const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t) * 8;
+  const int side_full = meta[0];
+  const int n_side_tiles = min(meta[1], p.side_tiles_cap);
+  const int win_tile_lo = meta[4];
+  const int n_tiles = n_side_tiles + (meta[5] - win_tile_lo);
+  const int row = t * kBM + tid;  // this thread's query position
+  const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
+
+  auto load_k = [&](int j) {
+    const int st = j & 1;
+    mbar_expect_tx(bar_k + st, NB * kTileBlockBytes);
+    const bool side = j < n_side_tiles;
+    const int y = side ? j * kBN : (win_tile_lo + (j - n_side_tiles)) * kBN;
+    for (int nb = 0; nb < NB; ++nb)
+      tma_load_3d(sK + (st * NB + nb) * kTileBlockBytes, side ? &mapKs : &mapK, bar_k + st,
+                  nb * 64, y, kv_plane);
+  };
+  auto load_v = [&](int j) {
+    const int st = j & 1;
+    mbar_expect_tx(bar_v + st, NB * kTileBlockBytes);
+    const bool side = j < n_side_tiles;
+    const int y = side ? j * kBN : (win_tile_lo + (j - n_side_tiles)) * kBN;
+    for (int nb = 0; nb < NB; ++nb)
+      tma_load_3d(sV + (st * NB + nb) * kTileBlockBytes, side ? &mapVs : &mapV, bar_v + st,
+                  nb * 64, y, kv_plane);
+  };
+  constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+  constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+  auto issue_s = [&](int j) {
+    const int st = j & 1;
+    const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * NB * kTileBlockBytes);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k) {
+      const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
+      umma_ss(tmem + tmem_S0 + st * 128, make_smem_desc(qa + off, 16, 1024),
+              make_smem_desc(ka + off, 16, 1024), idesc_s, k > 0);
+    }
+    tc_commit(bar_s + st);
+  };
+  auto issue_pv = [&](int j) {
+    const int st = j & 1;
+    const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * NB * kTileBlockBytes);
+#pragma unroll
+    for (int k = 0; k < kBN / 16; ++k) {
+      const uint32_t aoff = (k / 4) * kTileBlockBytes + (k % 4) * 32;
+      umma_ss(tmem + tmem_O, make_smem_desc(pa + aoff, 16, 1024),
+              make_smem_desc(va + k * 2048, kTileBlockBytes, 1024), idesc_o, (j > 0 || k > 0));
+    }
+    tc_commit(bar_o);
+  };
+  bool ok = true;
+  auto wait = [&](uint64_t* bar, uint32_t parity) {
+    if (!mbar_wait(bar, parity, abort_flag)) {
+      if (ok) set_status(p.status, SEPLLM_TIMEOUT);
+      ok = false;
+    }
+  };
+
+  if (leader) {
+    mbar_expect_tx(bar_q, NB * kTileBlockBytes);
+    for (int nb = 0; nb < NB; ++nb)
+      tma_load_3d(sQ + nb * kTileBlockBytes, &mapQ, bar_q, nb * 64, t * kBM, q_plane);
+    load_k(0);
+    load_v(0);
+    if (n_tiles > 1) load_k(1);
+    wait(bar_q, 0);
+    wait(bar_k + 0, 0);
+    tc_fence_after();
+    issue_s(0);
+  }
+
+  float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
+  float l_sum = 0.f;
+  uint32_t sreg[4][32];
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int st = j & 1;
+    wait(bar_s + st, (j >> 1) & 1);
+    tc_fence_after();
+    if (leader) {
+      if (j + 2 < n_tiles) load_k(j + 2);  // S(j) is complete, its K stage is free
+      if (j + 1 < n_tiles) {
+        wait(bar_k + ((j + 1) & 1), ((j + 1) >> 1) & 1);
+        tc_fence_after();
+        issue_s(j + 1);
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_ld32(tmem_row + tmem_S0 + st * 128 + c * 32, sreg[c]);
+    tmem_ld_wait();
+
+    // kept columns of this tile for this row: [c_lo, c_hi)
+    const bool side = j < n_side_tiles;
+    int c_lo = 0, c_hi = kBN;
+    bool need_mask;
+    if (side) {
+      c_hi = lim_i - j * kBN;
+      need_mask = (j >= side_full);
+    } else {
+      const int key0 = (win_tile_lo + (j - n_side_tiles)) * kBN;
+      c_hi = row - key0 + 1;
+      c_lo = row - p.n_neighbor + 1 - key0;
+      need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
+    }
+    float mx = -INFINITY;
+    if (need_mask) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int col = c * 32 + e;
+          float s = __uint_as_float(sreg[c][e]) * p.scale_log2;
+          s = (col >= c_lo && col < c_hi) ? s : -INFINITY;
+          sreg[c][e] = __float_as_uint(s);
+          mx = fmaxf(mx, s);
+        }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float s = __uint_as_float(sreg[c][e]) * p.scale_log2;
+          sreg[c][e] = __float_as_uint(s);
+          mx = fmaxf(mx, s);
+        }
+    }
+    // lazy rescale: move the reference only when the maximum grew by more than 2^8
+    float corr = 1.f;
+    bool rescale = false;
+    if (mx > m_ref + 8.f) {
+      corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
+      m_ref = mx;
+      rescale = true;
+    }
+    const float m_eff = (m_ref == -INFINITY) ? 0.f : m_ref;
+    float psum = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const float p0 = ex2(__uint_as_float(sreg[c][e]) - m_eff);
+        const float p1 = ex2(__uint_as_float(sreg[c][e + 1]) - m_eff);
+        psum += p0 + p1;
+        sreg[c][e >> 1] = pack_bf16(p0, p1);
+      }
+    l_sum = l_sum * corr + psum;
+
+    // PV(j-1) must be complete before O is rescaled and before P is overwritten
+    if (j > 0) {
+      wait(bar_o, (j - 1) & 1);
+      tc_fence_after();
+    }
+    __syncwarp();
+    if (leader && j + 1 < n_tiles) load_v(j + 1);  // PV(j-1) is complete, its V stage is free
+    if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+      uint32_t oreg[32];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        tmem_ld32(tmem_row + tmem_O + c * 32, oreg);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * corr);
+        tmem_st32(tmem_row + tmem_O + c * 32, oreg);
+      }
+      tmem_st_wait();
+    }
+    // P row -> shared memory, bf16, in the swizzled K-major layout the MMA reads
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const int chunk16 = c * 4 + q4;  // 16-byte chunk (8 keys) within the row of 128 keys
+        const uint4 val = make_uint4(sreg[c][q4 * 4 + 0], sreg[c][q4 * 4 + 1], sreg[c][q4 * 4 + 2],
+                                     sreg[c][q4 * 4 + 3]);
+        *reinterpret_cast<uint4*>(sP + (chunk16 >> 3) * kTileBlockBytes +
+                                  swz128(tid, chunk16 & 7)) = val;
+      }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (leader) {
+      tc_fence_after();
+      wait(bar_v + st, (j >> 1) & 1);
+      issue_pv(j);
+    }
+  }
+
+  wait(bar_o, (n_tiles - 1) & 1);
+  tc_fence_after();
+  __syncwarp();
+  const float inv_l = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+  if (row < p.L) p.LSE[size_t(q_plane) * p.L + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+  __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * D;
+#pragma unroll
+  for (int c = 0; c < D / 32; ++c) {
+    uint32_t oreg[32];
+    tmem_ld32(tmem_row + tmem_O + c * 32, oreg);
+    tmem_ld_wait();
+    if (row < p.L) {
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint4 val;
+        val.x = pack_bf16(__uint_as_float(oreg[q4 * 8 + 0]) * inv_l, __uint_as_float(oreg[q4 * 8 + 1]) * inv_l);
+        val.y = pack_bf16(__uint_as_float(oreg[q4 * 8 + 2]) * inv_l, __uint_as_float(oreg[q4 * 8 + 3]) * inv_l);
+        val.z = pack_bf16(__uint_as_float(oreg[q4 * 8 + 4]) * inv_l, __uint_as_float(oreg[q4 * 8 + 5]) * inv_l);
+        val.w = pack_bf16(__uint_as_float(oreg[q4 * 8 + 6]) * inv_l, __uint_as_float(oreg[q4 * 8 + 7]) * inv_l);
+        *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
+  if (!d || !id) return SEPLLM_INVALID_ARG;
+  if (d->B <= 0 || d->Hq <= 0 || d->Hkv <= 0 || d->L <= 0 || d->Hq % d->Hkv != 0)
+    return SEPLLM_INVALID_ARG;
+  if (id->B != d->B || id->L != d->L || id->n_neighbor < 1 || id->n_init < 0 || id->side_cap <= 0)
+    return SEPLLM_INVALID_ARG;
+  if (d->d != 64 && d->d != 128) return SEPLLM_UNSUPPORTED;
+  if (id->BM != kBM || id->BN != kBN) return SEPLLM_UNSUPPORTED;
+  if (d->grad_dtype != 0 && d->grad_dtype != 1) return SEPLLM_INVALID_ARG;
+  if (d->Hq > 65535 || d->B > 65535) return SEPLLM_UNSUPPORTED;
+  return SEPLLM_OK;
+}
+
+AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
+  AttnLayout a;
+  a.cap_pad = (id->side_cap + 127) / 128 * 128;
+  const size_t side_bytes = align_up(size_t(d->B) * d->Hkv * a.cap_pad * d->d * 2);
+  a.off_ks = kAlign;
+  a.off_vs = a.off_ks + side_bytes;
+  a.fwd_bytes = a.off_vs + side_bytes;
+  a.off_delta = a.fwd_bytes;
+  a.off_dks = a.off_delta + align_up(size_t(d->B) * d->Hq * d->L * sizeof(float));
+  const size_t side_grad = align_up(size_t(d->B) * d->Hkv * a.cap_pad * d->d * sizeof(float));
+  a.off_dvs = a.off_dks + side_grad;
+  a.bwd_bytes = a.off_dvs + side_grad;
+  return a;
+}
+
+void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
+                   const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
+                   void* Ks, void* Vs, cudaStream_t stream) {
+  if (d->d == 64) {
+    constexpr int RPB = 256 / (64 / 8);
+    gather_side_kv<64><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
+        n_side, d->L, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
+        static_cast<__nv_bfloat16*>(Vs));
+  } else {
+    constexpr int RPB = 256 / (128 / 8);
+    gather_side_kv<128><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
+        n_side, d->L, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
+        static_cast<__nv_bfloat16*>(Vs));
+  }
+}
+
+template <int D>
+static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_desc* id,
+                                const sepllm_index_header& ih, const void* Q, const void* K,
+                                const void* V, const uint8_t* index, void* O, float* LSE,
+                                uint8_t* ws, cudaStream_t stream) {
+  const AttnLayout lay = attn_layout(d, id);
+  __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(ws + lay.off_ks);
+  __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(ws + lay.off_vs);
+  const int32_t* side_pos = reinterpret_cast<const int32_t*>(index + ih.off_side_pos);
+  const int32_t* n_side = reinterpret_cast<const int32_t*>(index + ih.off_n_side);
+  launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
+
+  CUtensorMap mq, mk, mv, mks, mvs;
+  sepllm_status st;
+  const int64_t L = d->L;
+  if ((st = make_tile_map(&mq, Q, D, L, int64_t(d->B) * d->Hq, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mk, K, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mv, V, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mks, Ks, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
+                          int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mvs, Vs, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
+                          int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
+
+  FwdParams p;
+  p.lim = reinterpret_cast<const int32_t*>(index + ih.off_lim);
+  p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
+  p.O = static_cast<__nv_bfloat16*>(O);
+  p.LSE = LSE;
+  p.status = reinterpret_cast<int32_t*>(ws);
+  p.L = d->L;
+  p.T = ih.n_tiles;
+  p.Hq = d->Hq;
+  p.Hkv = d->Hkv;
+  p.n_neighbor = id->n_neighbor;
+  p.side_cap = id->side_cap;
+  p.side_tiles_cap = lay.cap_pad / 128;
+  const float scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
+  p.scale_log2 = scale * 1.4426950408889634f;
+  const uint32_t smem = FwdSmem<D>::kRequest;
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_kernel<D>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  attn_fwd_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), 128, smem, stream>>>(mq, mk, mv, mks, mvs, p);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  return SEPLLM_OK;
+}
+
+}  // namespace sepllm
+
+using namespace sepllm;
+
+extern "C" sepllm_status sepllm_attn_fwd(const sepllm_attn_desc* desc,
+                                         const sepllm_index_desc* idesc, const void* Q,
+                                         const void* K, const void* V, const void* index, void* O,
+                                         float* LSE, void* workspace, void* stream_) {
+  sepllm_status st = check_attn(desc, idesc);
+  if (st != SEPLLM_OK) return st;
+  if (!Q || !K || !V || !index || !O || !LSE || !workspace) return SEPLLM_INVALID_ARG;
+  if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
+      !aligned(LSE, 4) || !aligned(index, kAlign) || !aligned(workspace, kAlign))
+    return SEPLLM_INVALID_ARG;
+  sepllm_index_header ih;
+  if ((st = fill_index_header(idesc, &ih)) != SEPLLM_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
+  if (desc->d == 64)
+    return launch_fwd<64>(desc, idesc, ih, Q, K, V, static_cast<const uint8_t*>(index), O, LSE, ws,
+                          stream);
+  return launch_fwd<128>(desc, idesc, ih, Q, K, V, static_cast<const uint8_t*>(index), O, LSE, ws,
+                         stream);
+}

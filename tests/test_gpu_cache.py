@@ -120,8 +120,8 @@ def test_cache_medium_periodic():
 def test_cache_full_size_streaming_workload():
     """The streaming-decode workload's shapes: 32 sequences, 8 kv heads, c = 3332."""
     c = inputs.DECODE_CONFIG
-    gc, oc = _drive(c["B"], c["Hkv"], c["Hq"], c["d"], c["a"], c["s"], c["w"], c["c"], steps=5600,
-                    rho=c["rho"], seed=c["seed"], check_every=2800, pool=256)
+    gc, oc = _drive(c["B"], c["Hkv"], c["Hq"], c["d"], c["a"], c["s"], c["w"], c["c"], steps=6200,
+                    rho=c["rho"], seed=c["seed"], check_every=3100, pool=256)
     assert all(x.compactions >= 2 for x in oc)
 
 

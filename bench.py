@@ -1,0 +1,471 @@
+#!/usr/bin/env python
+"""Benchmark of the SepLLM attention hot path on B200.
+
+One step = the whole training-side hot path on one batch of synthetic input:
+sepllm_build_index -> sepllm_attn_fwd -> sepllm_attn_bwd.  The headline value is
+effective TFLOP/s on kept (query, key) pairs, 14*d flops per pair and query head
+(4*d forward, 10*d backward).  The streaming path (cache update + decode) and the
+index builder on a long id stream are measured in the same run and reported under
+"decode" and "index" with their own HBM rooflines.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+    python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+With N > 1 (torchrun) every rank runs its own copy of the workload (independent
+sequences; the path has no exchange step) and rank 0 reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2412_12094_b200 import inputs  # noqa: E402
+
+METRIC = "SepAttn fwd+bwd effective TFLOP/s (kept pairs)"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# ---------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(device_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.strip().split(", ") for r in open(self.tmp.name) if r.strip()]
+        os.unlink(self.tmp.name)
+        sm, reasons = [], set()
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                out["sm_max_mhz"] = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.strip().lower() == "active":
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(cfg, heads: int, prefix: int):
+    """Times the fp64 oracle (forward + backward) on the first `prefix` tokens of `heads`
+    query heads of the workload; returns (effective TFLOP/s, seconds, cores, description)."""
+    from threadpoolctl import threadpool_info
+    from oracle import sepllm_oracle as orc
+    L = min(prefix, cfg["L"])
+    ids = inputs.token_ids(cfg["seed"], 1, cfg["L"], cfg["rho"], cfg["structure"])[:, :L]
+    f = np.isin(ids[0], inputs.SEP_IDS)
+    d = cfg["d"]
+    G = cfg["Hq"] // cfg["Hkv"]
+    Q = inputs.normal_bf16(cfg["seed"], 1, (heads, L, d)).double().numpy()
+    K = inputs.normal_bf16(cfg["seed"], 2, (heads, L, d)).double().numpy()
+    V = inputs.normal_bf16(cfg["seed"], 3, (heads, L, d)).double().numpy()
+    dO = inputs.normal_bf16(cfg["seed"], 4, (heads, L, d)).double().numpy()
+    pairs = orc.kept_pairs(f, cfg["n_init"], cfg["n_neighbor"])
+    t0 = time.perf_counter()
+    M = orc.mask_matrix(f, cfg["n_init"], cfg["n_neighbor"])
+    for h in range(heads):
+        orc.attn_bwd_head(Q[h], K[h // G], V[h // G], dO[h], M)
+    dt = time.perf_counter() - t0
+    cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    tflops = 14.0 * d * pairs * heads / dt / 1e12
+    return tflops, dt, cores, f"fwd+bwd of {heads} query head(s) on the first {L} tokens of the workload"
+
+
+# ---------------------------------------------------------------------------- GPU arm
+class Workload:
+    def __init__(self, name: str, rank: int, device: torch.device):
+        from paper_2412_12094_b200 import api
+        self.api = api
+        cfg = dict(inputs.CONFIGS[name])
+        cfg["seed"] = cfg["seed"] + 1000 * rank
+        self.cfg, self.name, self.device = cfg, name, device
+        B, Hq, Hkv, L, d = cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["L"], cfg["d"]
+        self.ids_h = torch.from_numpy(inputs.token_ids(cfg["seed"], B, L, cfg["rho"], cfg["structure"])).pin_memory()
+        Q, K, V, dO = inputs.qkv_do(cfg["seed"], B, Hq, Hkv, L, d)
+        self.host = [t.pin_memory() for t in (Q, K, V, dO)]
+        self.ids = self.ids_h.to(device)
+        self.Q, self.K, self.V, self.dO = (t.to(device) for t in self.host)
+        self.idesc = api.IndexDesc(B, L, cfg["n_init"], cfg["n_neighbor"], len(inputs.SEP_IDS), 128, 128, L)
+        ib, sb = api.sepllm_index_bytes(self.idesc)
+        self.index = api.alloc_bytes(ib)
+        self.scratch = api.alloc_bytes(sb)
+        self.fdesc = api.AttnDesc(B, Hq, Hkv, d, L, 0.0, 0)
+        self.bdesc = api.AttnDesc(B, Hq, Hkv, d, L, 0.0, 0)
+        self.bdesc.flags = api.SIDE_READY          # backward reuses the forward's side K/V
+        _, bb = api.sepllm_attn_workspace_bytes(self.fdesc, self.idesc)
+        self.ws = api.alloc_bytes(bb)
+        self.O = torch.empty_like(self.Q)
+        self.LSE = torch.empty((B, Hq, L), dtype=torch.float32, device=device)
+        self.dQ = torch.empty_like(self.Q)
+        self.dK = torch.empty_like(self.K)
+        self.dV = torch.empty_like(self.V)
+        self.out_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (self.O, self.dQ, self.dK, self.dV)]
+        self.launches_per_step = 3 + 2 + 4
+
+    def step(self):
+        api = self.api
+        api.sepllm_build_index(self.idesc, self.ids, inputs.SEP_IDS, self.index, self.scratch)
+        api.sepllm_attn_fwd(self.fdesc, self.idesc, self.Q, self.K, self.V, self.index, self.O, self.LSE, self.ws)
+        api.sepllm_attn_bwd(self.bdesc, self.idesc, self.dO, self.Q, self.K, self.V, self.O, self.LSE,
+                            self.index, self.dQ, self.dK, self.dV, self.ws)
+
+    def step_e2e(self):
+        self.ids.copy_(self.ids_h, non_blocking=True)
+        for dst, src in zip((self.Q, self.K, self.V, self.dO), self.host):
+            dst.copy_(src, non_blocking=True)
+        self.step()
+        for dst, src in zip(self.out_h, (self.O, self.dQ, self.dK, self.dV)):
+            dst.copy_(src, non_blocking=True)
+
+    def e2e_bytes(self):
+        h2d = self.ids_h.numel() * 4 + sum(t.numel() * 2 for t in self.host)
+        d2h = sum(t.numel() * 2 for t in self.out_h)
+        return h2d, d2h
+
+    def kept_pairs(self):
+        torch.cuda.synchronize()
+        idx = self.api.read_index(self.index)
+        assert idx["header"].status == 0
+        assert self.api.sepllm_last_device_status(self.ws) == 0
+        total = idx["tile_meta"][:, :, 6].astype(np.int64).sum()
+        side = idx["lim"].astype(np.int64).sum()
+        return int(total), int(side)
+
+
+def timed(fn, steps, warmup, dist_barrier):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    dist_barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return e0.elapsed_time(e1) / 1e3
+
+
+def kernel_times(wl: Workload, steps: int):
+    """Per-kernel average durations (seconds) from events the library records between its launches."""
+    def mk(n):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in evs:
+            e.record()           # creates the handle
+        return evs
+    fsets = [mk(3) for _ in range(steps)]
+    bsets = [mk(6) for _ in range(steps)]
+    isets = [mk(2) for _ in range(steps)]
+    torch.cuda.synchronize()
+    api = wl.api
+    for s in range(steps):
+        isets[s][0].record()
+        api.sepllm_build_index(wl.idesc, wl.ids, inputs.SEP_IDS, wl.index, wl.scratch)
+        isets[s][1].record()
+        wl.fdesc.set_events(fsets[s])
+        api.sepllm_attn_fwd(wl.fdesc, wl.idesc, wl.Q, wl.K, wl.V, wl.index, wl.O, wl.LSE, wl.ws)
+        wl.bdesc.set_events(bsets[s])
+        api.sepllm_attn_bwd(wl.bdesc, wl.idesc, wl.dO, wl.Q, wl.K, wl.V, wl.O, wl.LSE, wl.index,
+                            wl.dQ, wl.dK, wl.dV, wl.ws)
+    torch.cuda.synchronize()
+    wl.fdesc.set_events(None)
+    wl.bdesc.set_events(None)
+
+    def avg(sets, i):
+        return sum(s[i].elapsed_time(s[i + 1]) for s in sets) / len(sets) / 1e3
+    return {
+        "build_index (3 kernels)": avg(isets, 0),
+        "gather_side_kv": avg(fsets, 0),
+        "attn_fwd_kernel": avg(fsets, 1),
+        "bwd_delta": avg(bsets, 1),
+        "bwd_dq_kernel": avg(bsets, 2),
+        "bwd_dkv_kernel<side>": avg(bsets, 3),
+        "bwd_dkv_kernel<window>": avg(bsets, 4),
+    }
+
+
+def bench_decode(device, peaks, steps=4096):
+    """Streaming workload: cache update + decode per step at the full cache shape."""
+    from paper_2412_12094_b200 import api
+    c = inputs.DECODE_CONFIG
+    B, Hq, Hkv, d = c["B"], c["Hq"], c["Hkv"], c["d"]
+    desc = api.CacheDesc(B, Hkv, Hq, d, c["a"], c["s"], c["w"], c["c"])
+    sb, kb = api.sepllm_cache_bytes(desc)
+    state = api.alloc_bytes(sb)
+    Kc = torch.zeros(kb // 2, dtype=torch.bfloat16, device=device)
+    Vc = torch.zeros(kb // 2, dtype=torch.bfloat16, device=device)
+    ws = api.alloc_bytes(api.sepllm_decode_workspace_bytes(desc))
+    api.sepllm_cache_init(desc, state)
+    pool = 256
+    warm = 12000                      # enough tokens to fill the separator cache (s / rho plus slack)
+    T = warm + steps
+    ids = inputs.decode_stream_ids(c["seed"], B, T, c["rho"])
+    ids_d = torch.from_numpy(np.ascontiguousarray(ids.T)).to(device)
+    kp, vp, qp = (t.to(device) for t in inputs.decode_kv_pool(c["seed"], pool, B, Hkv, Hq, d))
+    o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=device)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=device)
+
+    def step(t):
+        api.sepllm_cache_update(desc, state, Kc, Vc, ids_d[t], inputs.SEP_IDS, kp[t % pool], vp[t % pool])
+        api.sepllm_decode(desc, 0.0, qp[t % pool], state, Kc, Vc, o, lse, ws)
+
+    for t in range(warm):
+        step(t)
+    torch.cuda.synchronize()
+    st0 = api.read_cache_state(state)
+    # bookkeeping of Size_run per step (sizes only) for the byte count
+    f = np.isin(ids, inputs.SEP_IDS)
+    size_sep = st0["size_sep"].astype(np.int64).copy()
+    size_win = st0["size_win"].astype(np.int64).copy()
+    size_init = st0["size_init"].astype(np.int64)
+    rows = 0
+    # the window's separator flags are needed to know how many move at a compaction
+    win_flags = [list(f[b, warm - size_win[b]:warm]) for b in range(B)]
+    for t in range(warm, T):
+        for b in range(B):
+            win_flags[b].append(bool(f[b, t]))
+            if size_init[b] + size_sep[b] + len(win_flags[b]) == c["c"]:
+                n_past = len(win_flags[b]) - c["w"]
+                size_sep[b] = min(c["s"], size_sep[b] + sum(win_flags[b][:n_past]))
+                win_flags[b] = win_flags[b][n_past:]
+            rows += size_init[b] + size_sep[b] + len(win_flags[b])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(warm, T):
+        step(t)
+    e1.record()
+    torch.cuda.synchronize()
+    assert api.sepllm_last_device_status(state) == 0
+    st1 = api.read_cache_state(state)
+    assert (st1["size_sep"] == size_sep).all() and (st1["size_win"] == [len(w) for w in win_flags]).all()
+    sec = e0.elapsed_time(e1) / 1e3
+    bytes_total = rows * Hkv * d * 2 * 2          # K and V rows of every retained entry, every kv head
+    gbs = bytes_total / sec / 1e9
+    return {"workload": "B32 Hq32 Hkv8 d128 a4 s1024 w256 c3332, update+decode per step",
+            "steps": steps, "us_per_step": sec / steps * 1e6, "avg_size_run": rows / steps / B,
+            "bytes_per_step": bytes_total / steps, "achieved_gbs": gbs,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None},
+            "tokens_per_s": B * steps / sec, "gpu_launches": 4 * steps}
+
+
+def bench_index_stream(device, peaks, reps=20):
+    from paper_2412_12094_b200 import api
+    c = inputs.DECODE_CONFIG
+    B, L = c["B"], c["stream_len"]
+    ids = torch.from_numpy(inputs.decode_stream_ids(c["seed"], B, L, c["rho"])).to(device)
+    desc = api.IndexDesc(B, L, 4, 256, len(inputs.SEP_IDS), 128, 128, L // 4)
+    ib, sb = api.sepllm_index_bytes(desc)
+    index, scratch = api.alloc_bytes(ib), api.alloc_bytes(sb)
+    for _ in range(3):
+        api.sepllm_build_index(desc, ids, inputs.SEP_IDS, index, scratch)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        api.sepllm_build_index(desc, ids, inputs.SEP_IDS, index, scratch)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) / 1e3 / reps
+    n_side = int(api.read_index(index)["n_side"].astype(np.int64).sum())
+    T = (L + 127) // 128
+    algo = 4 * B * L + 4 * B * (L + 1) + 4 * B * L + 4 * n_side + 32 * B * T
+    gbs = algo / sec / 1e9
+    return {"workload": "32 x 2^20 token ids", "us": sec * 1e6, "bytes": algo,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_long_r10", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--no-extras", action="store_true", help="skip the decode / index-stream / e2e / CPU legs")
+    ap.add_argument("--cpu-prefix", type=int, default=8192)
+    ap.add_argument("--cpu-heads", type=int, default=4)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = inputs.CONFIGS[args.workload]
+    config = {"workload": f"{args.workload}: B{cfg['B']} Hq{cfg['Hq']} Hkv{cfg['Hkv']} d{cfg['d']} L{cfg['L']} "
+                          f"n_init{cfg['n_init']} n_neighbor{cfg['n_neighbor']} sep_rate{cfg['rho']} "
+                          f"({cfg['structure']}), fwd+bwd incl. index build",
+              "l2": "inputs larger than L2 (no flush)", "replicas": world}
+
+    if args.impl == "reference":
+        # the CPU oracle, as it stands, on a bounded sample; rank 0 only
+        if rank != 0:
+            return
+        vals, secs = [], []
+        for _ in range(args.warmup):
+            oracle_sample(cfg, 1, min(args.cpu_prefix, 2048))
+        for _ in range(args.steps):
+            v, dt, cores, what = oracle_sample(cfg, 1, min(args.cpu_prefix, 4096))
+            vals.append(v)
+            secs.append(dt)
+        val = sum(v * s for v, s in zip(vals, secs)) / sum(secs)   # time-weighted mean
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+        def barrier():
+            dist.barrier()
+    else:
+        dist = None
+
+        def barrier():
+            pass
+
+    peaks = load_peaks()
+    wl = Workload(args.workload, rank, device)
+    wl.step()
+    pairs, side_pairs = wl.kept_pairs()
+    d, Hq = cfg["d"], cfg["Hq"]
+    flops_step = 14.0 * d * pairs * Hq            # pairs is summed over the batch already
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    sec = timed(wl.step, args.steps, args.warmup, barrier)
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([sec], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+        fl = torch.tensor([flops_step], device=device, dtype=torch.float64)
+        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
+        flops_total_step = float(fl.item())
+    else:
+        flops_total_step = flops_step
+    value = flops_total_step * args.steps / sec / 1e12
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": config, "gpu_launches": wl.launches_per_step * args.steps,
+           "kept_pairs": pairs, "frac_of_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
+           "peaks": {k: peaks[k] for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}}
+    if clocks is not None:
+        out["clocks"] = clocks
+
+    # per-kernel durations and the roofline of the dominant kernel (rank 0's replica)
+    kt = kernel_times(wl, min(args.steps, 10))
+    win_pairs = pairs - side_pairs
+    kflops = {
+        "attn_fwd_kernel": 4.0 * d * pairs * Hq,
+        "bwd_dq_kernel": 6.0 * d * pairs * Hq,
+        "bwd_dkv_kernel<side>": 8.0 * d * side_pairs * Hq,
+        "bwd_dkv_kernel<window>": 8.0 * d * win_pairs * Hq,
+    }
+    tot = sum(kt.values())
+    out["kernels"] = {k: {"ms": v * 1e3, "share": v / tot,
+                          **({"tflops": kflops[k] / v / 1e12} if k in kflops and v > 0 else {})}
+                      for k, v in kt.items()}
+    dom = max(kflops, key=lambda k: kt[k])
+    ach = kflops[dom] / kt[dom] / 1e12
+    out["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                       "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                       "peak_kind": f"bf16 sustained, {peaks['source']}",
+                       "flops_per_launch": kflops[dom]}
+
+    if not args.no_extras:
+        # end to end: host buffers in, results back, copies inside the timed region
+        sec_e = timed(wl.step_e2e, max(2, args.steps // 2), 1, barrier)
+        if world > 1:
+            t = torch.tensor([sec_e], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            sec_e = float(t.item())
+        h2d, d2h = wl.e2e_bytes()
+        out["e2e"] = {"value": flops_total_step * max(2, args.steps // 2) / sec_e / 1e12, "unit": UNIT,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "ms_per_step": sec_e / max(2, args.steps // 2) * 1e3}
+        if rank == 0:
+            del wl
+            torch.cuda.empty_cache()
+            out["decode"] = bench_decode(device, peaks)
+            out["index"] = bench_index_stream(device, peaks)
+            if world == 1:
+                v, dt, cores, what = oracle_sample(cfg, args.cpu_heads, args.cpu_prefix)
+                out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                       "sample": what, "seconds": dt}
+    if world > 1:
+        barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

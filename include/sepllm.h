@@ -59,11 +59,24 @@ typedef struct {
 } sepllm_index_desc;
 
 /* scale = 0 means 1/sqrt(d) (Eq. 1).  grad_dtype: 0 = bf16, 1 = fp32 outputs
- * for dQ, dK, dV. */
+ * for dQ, dK, dV.
+ * flags: SEPLLM_ATTN_SIDE_READY = the workspace already holds the side K/V rows
+ *   gathered from these K, V by an earlier attention call on the same workspace
+ *   (a backward given the forward's workspace); the call then skips its gather.
+ * events / n_events: optional host array of cudaEvent_t handles (NULL / 0 = off).
+ *   The call records events[0] on `stream` before its first launch and
+ *   events[i] after its i-th launch, for as many as the array holds, so a
+ *   caller can time each kernel.  Forward launches: 1 side gather, 2 attention.
+ *   Backward launches: 1 side gather, 2 Delta, 3 dQ, 4 dK/dV of side tiles,
+ *   5 dK/dV of window tiles.  A skipped gather still records its event. */
+#define SEPLLM_ATTN_SIDE_READY 1
 typedef struct {
   int32_t B, Hq, Hkv, d, L;
   float scale;
   int32_t grad_dtype;
+  int32_t flags;
+  void* const* events;
+  int32_t n_events;
 } sepllm_attn_desc;
 
 /* Streaming cache capacities in the paper's names (Section 3.3): a initial,

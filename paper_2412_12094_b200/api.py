@@ -22,9 +22,24 @@ class IndexDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("B", "L", "n_init", "n_neighbor", "n_sep", "BM", "BN", "side_cap")]
 
 
+SIDE_READY = 1
+
+
 class AttnDesc(C.Structure):
     _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32),
-                ("L", C.c_int32), ("scale", C.c_float), ("grad_dtype", C.c_int32)]
+                ("L", C.c_int32), ("scale", C.c_float), ("grad_dtype", C.c_int32),
+                ("flags", C.c_int32), ("events", C.POINTER(C.c_void_p)), ("n_events", C.c_int32)]
+
+    def set_events(self, events):
+        """events: torch.cuda.Event objects (timing enabled, recorded once so their handles
+        exist), or None to switch per-kernel timing off."""
+        if not events:
+            self.events, self.n_events, self._keep = None, 0, None
+            return
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        self._keep = arr
+        self.events = C.cast(arr, C.POINTER(C.c_void_p))
+        self.n_events = len(events)
 
 
 class CacheDesc(C.Structure):

@@ -27,6 +27,12 @@ __global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
                                int cap_pad, __nv_bfloat16* __restrict__ Ks,
                                __nv_bfloat16* __restrict__ Vs);
 
+// Records desc->events[i] on the stream if the caller asked for it.
+inline void record_event(const sepllm_attn_desc* d, int i, cudaStream_t stream) {
+  if (d->events && i < d->n_events && d->events[i])
+    cudaEventRecord(static_cast<cudaEvent_t>(d->events[i]), stream);
+}
+
 // Launches the gather of K/V rows at the side positions into Ks / Vs ([B][Hkv][cap_pad][d]).
 void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
                    const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,

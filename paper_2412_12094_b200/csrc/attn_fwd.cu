@@ -431,7 +431,10 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(ws + lay.off_vs);
   const int32_t* side_pos = reinterpret_cast<const int32_t*>(index + ih.off_side_pos);
   const int32_t* n_side = reinterpret_cast<const int32_t*>(index + ih.off_n_side);
-  launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
+  record_event(d, 0, stream);
+  if (!(d->flags & SEPLLM_ATTN_SIDE_READY))
+    launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
+  record_event(d, 1, stream);
 
   CUtensorMap mq, mk, mv, mks, mvs;
   sepllm_status st;
@@ -463,6 +466,7 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_kernel<D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   attn_fwd_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), 128, smem, stream>>>(mq, mk, mv, mks, mvs, p);
+  record_event(d, 2, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }

@@ -1,0 +1,69 @@
+"""sepllm_attn_bwd against the fp64 oracle's analytic gradients."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sepllm_oracle as orc
+from paper_2412_12094_b200 import api, inputs
+from tests._gpu_util import TOL_GRAD, assert_close, attn_bwd, attn_fwd, build_index, flags_of
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(B, Hq, Hkv, L, d, a, n, rho, seed, grad_dtype=0, ids=None, sep_ids=inputs.SEP_IDS):
+    if ids is None:
+        ids = inputs.token_ids(seed, B, L, rho, "iid")
+    Q, K, V, dO = inputs.qkv_do(seed, B, Hq, Hkv, L, d)
+    idesc, index = build_index(ids, sep_ids, a, n)
+    Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
+    O, LSE = attn_fwd(Qd, Kd, Vd, idesc, index)
+    dQ, dK, dV = attn_bwd(dOd, Qd, Kd, Vd, O, LSE, idesc, index, grad_dtype)
+    rq, rk, rv = orc.attn_bwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(),
+                              dO.double().numpy(), flags_of(ids, sep_ids), a, n)
+    assert_close(dQ.float().cpu().numpy(), rq, TOL_GRAD, "dQ")
+    assert_close(dK.float().cpu().numpy(), rk, TOL_GRAD, "dK")
+    assert_close(dV.float().cpu().numpy(), rv, TOL_GRAD, "dV")
+    return (Qd, Kd, Vd, dOd, O, LSE, idesc, index), (dQ, dK, dV)
+
+
+def test_bwd_tiny_config():
+    c = inputs.CONFIGS["tiny"]
+    _run(c["B"], c["Hq"], c["Hkv"], c["L"], c["d"], c["n_init"], c["n_neighbor"], c["rho"], c["seed"])
+
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 2, 2), (128, 4, 1), (128, 2, 2), (64, 4, 2)])
+@pytest.mark.parametrize("L,a,n", [(512, 4, 64), (300, 4, 64), (777, 3, 200), (129, 2, 128), (1000, 4, 1000)])
+def test_bwd_shapes(d, Hq, Hkv, L, a, n):
+    _run(2, Hq, Hkv, L, d, a, n, 0.15, 200 + L + d)
+
+
+def test_bwd_fp32_gradients_and_determinism():
+    args, (dQ, dK, dV) = _run(1, 4, 2, 900, 128, 4, 100, 0.2, 71, grad_dtype=1)
+    assert dQ.dtype == torch.float32
+    Qd, Kd, Vd, dOd, O, LSE, idesc, index = args
+    dQ2, dK2, dV2 = attn_bwd(dOd, Qd, Kd, Vd, O, LSE, idesc, index, 1)
+    assert torch.equal(dQ, dQ2) and torch.equal(dK, dK2) and torch.equal(dV, dV2)
+
+
+def test_bwd_special_masks():
+    L = 640
+    _run(1, 2, 1, L, 128, 0, L, 0.1, 81)                      # dense causal
+    _run(1, 2, 1, L, 64, 0, 100, 0.0, 82)                     # sliding window, empty side list
+    ids = np.full((1, L), inputs.SEP_IDS[0], dtype=np.int32)
+    _run(1, 2, 2, L, 64, 0, 1, 0.0, 83, ids=ids)              # every token a separator, n = 1
+    _run(1, 2, 2, 256, 64, 0, 1, 0.3, 84)                     # n = 1 with sparse separators
+
+
+def test_bwd_many_side_tiles():
+    _run(1, 4, 2, 3000, 128, 4, 300, 0.3, 91)
+    _run(1, 2, 2, 2500, 64, 4, 77, 0.4, 92)
+
+
+def test_bwd_dv_column_sums_property():
+    """Rows of A sum to one, so sum_j dV[j] equals the sum of dO over the queries of the group."""
+    args, (dQ, dK, dV) = _run(1, 4, 2, 1100, 64, 4, 128, 0.12, 93, grad_dtype=1)
+    dOd = args[3]
+    lhs = dV.double().sum(dim=2)                                  # [B][Hkv][d]
+    rhs = dOd.double().view(1, 2, 2, 1100, 64).sum(dim=(2, 3))
+    # bf16 rounding of P leaves each row sum of A off by ~1e-4; over 2200 rows that is ~1e-2 here
+    assert torch.allclose(lhs, rhs, atol=0.1, rtol=1e-3)

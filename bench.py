@@ -185,6 +185,17 @@ class Workload:
         return int(total), int(side)
 
 
+def aggregate(sec: float, work: float, device, dist=None):
+    """Whole-job figures from per-rank ones: time = max over ranks, work = sum over ranks."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return sec, work
+    t = torch.tensor([sec], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    w = torch.tensor([work], device=device, dtype=torch.float64)
+    dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(w.item())
+
+
 def timed(fn, steps, warmup, dist_barrier):
     for _ in range(warmup):
         fn()
@@ -400,15 +411,7 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     sec = timed(wl.step, args.steps, args.warmup, barrier)
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([sec], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
-        fl = torch.tensor([flops_step], device=device, dtype=torch.float64)
-        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
-        flops_total_step = float(fl.item())
-    else:
-        flops_total_step = flops_step
+    sec, flops_total_step = aggregate(sec, flops_step, device, dist)
     value = flops_total_step * args.steps / sec / 1e12
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -443,10 +446,7 @@ def main():
     if not args.no_extras:
         # end to end: host buffers in, results back, copies inside the timed region
         sec_e = timed(wl.step_e2e, max(2, args.steps // 2), 1, barrier)
-        if world > 1:
-            t = torch.tensor([sec_e], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            sec_e = float(t.item())
+        sec_e, _ = aggregate(sec_e, 0.0, device, dist)
         h2d, d2h = wl.e2e_bytes()
         out["e2e"] = {"value": flops_total_step * max(2, args.steps // 2) / sec_e / 1e12, "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

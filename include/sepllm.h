@@ -131,6 +131,28 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
                                  const int32_t* sep_ids, void* index, void* scratch,
                                  void* stream);
 
+/* Same result as sepllm_build_index, for callers that cannot hand over a scratch
+ * buffer because they cannot allocate device memory at the point of the call: a
+ * serving process whose memory pool is already fully handed out, a plugin or
+ * callback that runs where cudaMalloc is forbidden, or a latency-critical loop
+ * that must not take cudaMalloc's device-wide synchronisation.  (The paper has
+ * no counterpart; this is a packaging variant of the index build.)
+ * The scratch lives in a fixed 256 KB array inside the library image, present
+ * on every device that loads the library until the process exits.  Limit:
+ * B * ceil(L / 4096) <= 65536 chunks; beyond it the call returns
+ * SEPLLM_BUFFER_TOO_SMALL and launches nothing.  The call itself allocates
+ * nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ * The first call on each device looks up the array's device address; make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array: two calls whose kernels may overlap on the GPU (different streams
+ * without ordering, or different host threads) race on it and must be
+ * serialised by the caller.  Nothing in the array has to be zero on entry: every
+ * word a call reads it has written itself, so back-to-back calls are
+ * independent.  Other arguments and the written index are exactly those of
+ * sepllm_build_index. */
+sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc, const int32_t* token_ids,
+                                        const int32_t* sep_ids, void* index, void* stream);
+
 /* Workspace sizes for the attention calls (bytes; either pointer may be NULL). */
 sepllm_status sepllm_attn_workspace_bytes(const sepllm_attn_desc* desc,
                                           const sepllm_index_desc* idesc, size_t* fwd_bytes,

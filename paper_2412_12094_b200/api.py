@@ -62,7 +62,8 @@ class CacheHeader(C.Structure):
 
 
 EXPORTS = [
-    "sepllm_index_bytes", "sepllm_build_index", "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
+    "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_static",
+    "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
     "sepllm_decode_workspace_bytes", "sepllm_decode", "sepllm_last_device_status",
     "sepllm_status_string",
@@ -133,6 +134,16 @@ def sepllm_build_index(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index:
     assert n == desc.n_sep
     _check(lib().sepllm_build_index(C.byref(desc), _ptr(token_ids), p, _ptr(index), _ptr(scratch),
                                     _stream()), "sepllm_build_index")
+
+
+def sepllm_build_index_static(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index: torch.Tensor):
+    """Index build for callers that cannot allocate a scratch buffer: the library's own fixed
+    array is used instead (B * ceil(L/4096) <= 65536).  Calls that may overlap on the GPU must be
+    serialised by the caller; make the first call on a device outside any stream capture."""
+    arr, p, n = _sep_array(sep_ids)
+    assert n == desc.n_sep
+    _check(lib().sepllm_build_index_static(C.byref(desc), _ptr(token_ids), p, _ptr(index), _stream()),
+           "sepllm_build_index_static")
 
 
 def read_index(index: torch.Tensor) -> dict:

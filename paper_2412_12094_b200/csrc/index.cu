@@ -6,6 +6,8 @@
 //   2. index_scan  : chunk offset (sum of earlier chunk counts) + in-chunk prefix scan;
 //                    writes cnt, the shifted copy lim[i] = cnt[i-n+1], and side_pos
 //   3. index_tiles : per query tile metadata, side_pos tail fill, header
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sepllm {
@@ -251,6 +253,73 @@ extern "C" sepllm_status sepllm_build_index(const sepllm_index_desc* desc,
   int32_t* chunk_sums = static_cast<int32_t*>(scratch);
   SEPLLM_CUDA_TRY(cudaMemsetAsync(blob, 0, sizeof(sepllm_index_header), stream));
   dim3 grid(n_chunks, desc->B);
+  index_count<<<grid, kIdxThreads, 0, stream>>>(token_ids, desc->L, desc->n_init, sep, chunk_sums,
+                                                n_chunks);
+  index_scan<<<grid, kIdxThreads, 0, stream>>>(
+      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, chunk_sums, n_chunks,
+      desc->side_cap, reinterpret_cast<int32_t*>(blob + h.off_cnt),
+      reinterpret_cast<int32_t*>(blob + h.off_lim),
+      reinterpret_cast<int32_t*>(blob + h.off_side_pos),
+      reinterpret_cast<int32_t*>(blob + h.off_n_side), reinterpret_cast<int32_t*>(blob));
+  const int units = desc->B * h.n_tiles;
+  const int blocks = max(1, min(148 * 4, (units + 7) / 8));
+  index_tiles<<<blocks, 256, 0, stream>>>(h, blob);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  return SEPLLM_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Index build without caller-provided scratch
+// ---------------------------------------------------------------------------
+// Chunk sums for sepllm_build_index_static live in this fixed array instead of a caller buffer.
+// 65536 chunks of 4096 ids = 256 KB, held by every device that loads the library until exit.
+constexpr int kStaticChunks = 65536;
+static __device__ __align__(256) int32_t g_static_chunk_sums[kStaticChunks];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static int32_t* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the array on the current device.  The array's name is only a host-side
+// handle here, so the address is looked up once per device and cached.
+static sepllm_status static_chunk_sums(int32_t** out) {
+  int dev = -1;
+  SEPLLM_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return SEPLLM_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    SEPLLM_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_chunk_sums));
+    if (!p) return SEPLLM_CUDA_ERROR;
+    g_static_ptr[dev] = static_cast<int32_t*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc,
+                                                   const int32_t* token_ids,
+                                                   const int32_t* sep_ids, void* index,
+                                                   void* stream_) {
+  sepllm_index_header h;
+  sepllm_status st = fill_index_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  if (!token_ids || !index || (desc->n_sep > 0 && !sep_ids)) return SEPLLM_INVALID_ARG;
+  if (!aligned(index, kAlign) || !aligned(token_ids, 4)) return SEPLLM_INVALID_ARG;
+  if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
+  const int n_chunks = (desc->L + kIdxChunk - 1) / kIdxChunk;
+  if (static_cast<int64_t>(desc->B) * n_chunks > kStaticChunks) return SEPLLM_BUFFER_TOO_SMALL;
+  int32_t* chunk_sums = nullptr;
+  if ((st = static_chunk_sums(&chunk_sums)) != SEPLLM_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  SepIds sep;
+  sep.n = desc->n_sep;
+  for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k) sep.id[k] = (k < sep.n) ? sep_ids[k] : -1;
+  uint8_t* blob = static_cast<uint8_t*>(index);
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(blob, 0, sizeof(sepllm_index_header), stream));
+  dim3 grid(n_chunks, desc->B);
+  // index_count writes every chunk sum that index_scan reads, so nothing left in the array by an
+  // earlier call is ever used and nothing has to be cleared.
   index_count<<<grid, kIdxThreads, 0, stream>>>(token_ids, desc->L, desc->n_init, sep, chunk_sums,
                                                 n_chunks);
   index_scan<<<grid, kIdxThreads, 0, stream>>>(

@@ -82,6 +82,9 @@ CONFIGS = {
                        n_init=4, n_neighbor=256, seed=1002),
     "llama8b_prefill": dict(B=1, Hq=32, Hkv=8, d=128, L=8192, rho=0.10, structure="geometric",
                             n_init=4, n_neighbor=256, seed=1003),
+    # a shorter copy of the long-context shape, for profiler captures (inputs still exceed L2)
+    "llama8b_L16k_r10": dict(B=1, Hq=32, Hkv=8, d=128, L=16384, rho=0.10, structure="geometric",
+                             n_init=4, n_neighbor=512, seed=1008),
     "llama8b_long_r05": dict(B=1, Hq=32, Hkv=8, d=128, L=65536, rho=0.05, structure="geometric",
                              n_init=4, n_neighbor=512, seed=1004),
     "llama8b_long_r10": dict(B=1, Hq=32, Hkv=8, d=128, L=65536, rho=0.10, structure="geometric",

@@ -4,11 +4,11 @@
 //   side   entries [0, lim[i]) of the per-sequence side buffer (initial tokens and separators at
 //          distance >= n from the row), gathered once into contiguous K/V side buffers;
 //   window keys i-n < j <= i, read from K/V in place.
-// One CTA walks the side tiles and then the window tiles of its query tile: TMA brings 128-key
-// K/V tiles into shared memory, tcgen05 MMAs compute S = Q K^T into tensor memory, the CTA's 128
-// threads (one per query row, matching tensor-memory lanes) run the online softmax, P goes back
-// through shared memory as bf16 and a second MMA accumulates O += P V in tensor memory.  Only
-// tiles crossing lim[], the diagonal or the window's left edge are masked element by element.
+// A CTA walks the side tiles and then the window tiles of its query tiles: TMA brings 128-key
+// K/V tiles into shared memory, tcgen05 MMAs compute S = Q K^T into tensor memory, one thread
+// per query row (= tensor-memory lane) runs the online softmax, P returns to tensor memory as
+// bf16 and a second MMA accumulates O += P V there.  Only tiles crossing lim[], the diagonal or
+// the window's left edge are masked element by element.
 #include "attn_common.cuh"
 
 namespace sepllm {
@@ -81,18 +81,32 @@ gather_side_kv(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restr
 // ---------------------------------------------------------------------------
 // forward kernel
 // ---------------------------------------------------------------------------
+// One CTA works on two query tiles ("slots") that share their key tiles: two query heads of one
+// GQA group at the same tile position when the group size is even, else two adjacent tiles of
+// one head.  Twelve warps:
+//   warp 0      TMA producer: Q of both slots, then the K and V tiles through NST-stage rings
+//   warp 1      MMA issuer:   S_x = Q_x K^T and O_x += P_x V for both slots, all in tensor memory
+//   warps 4-7   softmax of slot 0, one thread per query row (= tensor-memory lane)
+//   warps 8-11  softmax of slot 1
+// P never touches shared memory: the softmax threads write it as packed bf16 over the first half
+// of their slot's S columns and the PV MMA takes its A operand from tensor memory.  The issuer
+// alternates slots, so one slot's softmax runs under the other slot's MMAs.
 template <int D>
-struct FwdSmem {
-  static constexpr int NB = D / 64;  // 64-column blocks per row
+struct FwdCfg {
+  static constexpr int NB = D / 64;                 // 64-column blocks per row
+  static constexpr int NST = (D == 128) ? 2 : 4;    // K and V ring depth
+  static constexpr uint32_t kTile = NB * kTileBlockBytes;
   static constexpr uint32_t kQ = 0;
-  static constexpr uint32_t kK = kQ + NB * kTileBlockBytes;
-  static constexpr uint32_t kV = kK + 2 * NB * kTileBlockBytes;
-  static constexpr uint32_t kP = kV + 2 * NB * kTileBlockBytes;
-  static constexpr uint32_t kBar = kP + 2 * kTileBlockBytes;
-  static constexpr uint32_t kTotal = kBar + 256;
-  // one CTA per SM: each CTA takes all 512 tensor-memory columns
-  static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
+  static constexpr uint32_t kK = kQ + 2 * kTile;
+  static constexpr uint32_t kV = kK + NST * kTile;
+  static constexpr uint32_t kBar = kV + NST * kTile;
+  static constexpr uint32_t kTotal = kBar + 512;
+  static constexpr uint32_t kRequest = kTotal + 1024;  // > half an SM: one CTA per SM owns all 512 TMEM columns
+  // tensor-memory columns
+  static constexpr uint32_t kS0 = 0, kS1 = 128, kO0 = 256, kO1 = 256 + D;
 };
+
+constexpr int kFwdThreads = 384;
 
 struct FwdParams {
   const int32_t* lim;        // [B][L]
@@ -100,45 +114,95 @@ struct FwdParams {
   __nv_bfloat16* O;
   float* LSE;
   int32_t* status;
-  int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap;
+  int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap, pair_heads;
   float scale_log2;
 };
 
+// D[tmem] (+)= A[tmem, packed bf16] * B[smem]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc,
+                                        uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKs,
                 const __grid_constant__ CUtensorMap mapVs, const FwdParams p) {
-  using SM = FwdSmem<D>;
-  constexpr int NB = SM::NB;
+  using C = FwdCfg<D>;
+  constexpr int NB = C::NB, NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* sQ = smem + SM::kQ;
-  uint8_t* sK = smem + SM::kK;
-  uint8_t* sV = smem + SM::kV;
-  uint8_t* sP = smem + SM::kP;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBar);
-  uint64_t* bar_q = bars + 0;
-  uint64_t* bar_k = bars + 1;  // [2]
-  uint64_t* bar_v = bars + 3;  // [2]
-  uint64_t* bar_s = bars + 5;  // [2]
-  uint64_t* bar_o = bars + 7;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+  uint8_t* sQ = smem + C::kQ;
+  uint8_t* sK = smem + C::kK;
+  uint8_t* sV = smem + C::kV;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
+  uint64_t* bar_q = bars;                   // [2]   Q of slot x landed
+  uint64_t* bar_s = bars + 2;               // [2]   S_x complete (and every earlier MMA)
+  uint64_t* bar_p = bars + 4;               // [2]   P_x written by its 128 softmax threads
+  uint64_t* bar_o = bars + 6;               //       every MMA of the CTA complete
+  uint64_t* bar_kf = bars + 8;              // [NST] K stage full
+  uint64_t* bar_ke = bar_kf + NST;          // [NST] K stage free
+  uint64_t* bar_vf = bar_ke + NST;          // [NST]
+  uint64_t* bar_ve = bar_vf + NST;          // [NST]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + 4 * NST);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const bool leader = (tid == 0);
-  const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
-  const int hq = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
-  const int q_plane = b * p.Hq + hq;
-  const int kv_plane = b * p.Hkv + hq / G;
 
-  if (leader) {
-    mbar_init(bar_q, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_k + i, 1); mbar_init(bar_v + i, 1); mbar_init(bar_s + i, 1); }
+  // the two slots of this CTA (slot 1 is never empty; slot 0 is when T is odd and tiles pair up)
+  int t_x[2], hq_x[2];
+  if (p.pair_heads) {
+    t_x[0] = t_x[1] = p.T - 1 - int(blockIdx.x);  // long tiles first
+    hq_x[0] = 2 * int(blockIdx.y);
+    hq_x[1] = hq_x[0] + 1;
+  } else {
+    t_x[1] = p.T - 1 - 2 * int(blockIdx.x);
+    t_x[0] = t_x[1] - 1;
+    hq_x[0] = hq_x[1] = int(blockIdx.y);
+  }
+  const int kv_plane = b * p.Hkv + hq_x[0] / G;
+  int side_full_x[2], ns_x[2], wlo_x[2], whi_x[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    if (t_x[x] >= 0) {
+      const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t_x[x]) * 8;
+      side_full_x[x] = meta[0];
+      ns_x[x] = min(meta[1], p.side_tiles_cap);
+      wlo_x[x] = meta[4];
+      whi_x[x] = meta[5];
+    } else {
+      side_full_x[x] = 0; ns_x[x] = 0; wlo_x[x] = wlo_x[1 - x]; whi_x[x] = wlo_x[x];
+    }
+  }
+  if (t_x[0] < 0) { wlo_x[0] = wlo_x[1]; whi_x[0] = wlo_x[1]; }
+  // key tiles of the CTA: side tiles [0, ns), then window tiles [wlo, whi)
+  const int ns = max(ns_x[0], ns_x[1]);
+  const int wlo = min(wlo_x[0], wlo_x[1]);
+  const int whi = max(whi_x[0], whi_x[1]);
+  const int n_tiles = ns + (whi - wlo);
+  auto active = [&](int x, int j) -> bool {
+    if (j < ns) return j < ns_x[x];
+    const int w = wlo + (j - ns);
+    return w >= wlo_x[x] && w < whi_x[x];
+  };
+
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_s + i, 1); mbar_init(bar_p + i, 128); }
     mbar_init(bar_o, 1);
+    for (int i = 0; i < NST; ++i) {
+      mbar_init(bar_kf + i, 1); mbar_init(bar_ke + i, 1); mbar_init(bar_vf + i, 1); mbar_init(bar_ve + i, 1);
+    }
     *abort_flag = 0;
     fence_mbar_init();
     tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
@@ -153,59 +217,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_row = tmem + (uint32_t(warp * 32) << 16);
-  const uint32_t tmem_S0 = 0, tmem_O = 256;
 
-  const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t) * 8;
-  const int side_full = meta[0];
-  const int n_side_tiles = min(meta[1], p.side_tiles_cap);
-  const int win_tile_lo = meta[4];
-  const int n_tiles = n_side_tiles + (meta[5] - win_tile_lo);
-  const int row = t * kBM + tid;  // this thread's query position
-  const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-
-  auto load_k = [&](int j) {
-    const int st = j & 1;
-    mbar_expect_tx(bar_k + st, NB * kTileBlockBytes);
-    const bool side = j < n_side_tiles;
-    const int y = side ? j * kBN : (win_tile_lo + (j - n_side_tiles)) * kBN;
-    for (int nb = 0; nb < NB; ++nb)
-      tma_load_3d(sK + (st * NB + nb) * kTileBlockBytes, side ? &mapKs : &mapK, bar_k + st,
-                  nb * 64, y, kv_plane);
-  };
-  auto load_v = [&](int j) {
-    const int st = j & 1;
-    mbar_expect_tx(bar_v + st, NB * kTileBlockBytes);
-    const bool side = j < n_side_tiles;
-    const int y = side ? j * kBN : (win_tile_lo + (j - n_side_tiles)) * kBN;
-    for (int nb = 0; nb < NB; ++nb)
-      tma_load_3d(sV + (st * NB + nb) * kTileBlockBytes, side ? &mapVs : &mapV, bar_v + st,
-                  nb * 64, y, kv_plane);
-  };
-  constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
-  constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
-  auto issue_s = [&](int j) {
-    const int st = j & 1;
-    const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * NB * kTileBlockBytes);
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k) {
-      const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-      umma_ss(tmem + tmem_S0 + st * 128, make_smem_desc(qa + off, 16, 1024),
-              make_smem_desc(ka + off, 16, 1024), idesc_s, k > 0);
-    }
-    tc_commit(bar_s + st);
-  };
-  auto issue_pv = [&](int j) {
-    const int st = j & 1;
-    const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * NB * kTileBlockBytes);
-#pragma unroll
-    for (int k = 0; k < kBN / 16; ++k) {
-      const uint32_t aoff = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-      umma_ss(tmem + tmem_O, make_smem_desc(pa + aoff, 16, 1024),
-              make_smem_desc(va + k * 2048, kTileBlockBytes, 1024), idesc_o, (j > 0 || k > 0));
-    }
-    tc_commit(bar_o);
-  };
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (!mbar_wait(bar, parity, abort_flag)) {
@@ -214,156 +226,203 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     }
   };
 
-  if (leader) {
-    mbar_expect_tx(bar_q, NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb)
-      tma_load_3d(sQ + nb * kTileBlockBytes, &mapQ, bar_q, nb * 64, t * kBM, q_plane);
-    load_k(0);
-    load_v(0);
-    if (n_tiles > 1) load_k(1);
-    wait(bar_q, 0);
-    wait(bar_k + 0, 0);
-    tc_fence_after();
-    issue_s(0);
-  }
-
-  float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
-  float l_sum = 0.f;
-  uint32_t sreg[4][32];
-
-  for (int j = 0; j < n_tiles; ++j) {
-    const int st = j & 1;
-    wait(bar_s + st, (j >> 1) & 1);
-    tc_fence_after();
-    if (leader) {
-      if (j + 2 < n_tiles) load_k(j + 2);  // S(j) is complete, its K stage is free
-      if (j + 1 < n_tiles) {
-        wait(bar_k + ((j + 1) & 1), ((j + 1) >> 1) & 1);
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 0 && lane == 0) {
+      // ---------------- TMA producer ----------------
+#pragma unroll
+      for (int x = 0; x < 2; ++x)
+        if (t_x[x] >= 0) {
+          mbar_expect_tx(bar_q + x, C::kTile);
+          for (int nb = 0; nb < NB; ++nb)
+            tma_load_3d(sQ + x * C::kTile + nb * kTileBlockBytes, &mapQ, bar_q + x, nb * 64,
+                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+        }
+      for (int j = 0; j < n_tiles; ++j) {
+        const int st = j % NST, use = j / NST;
+        const bool side = j < ns;
+        const int y = side ? j * kBN : (wlo + (j - ns)) * kBN;
+        if (use > 0) wait(bar_ke + st, (use - 1) & 1);
+        mbar_expect_tx(bar_kf + st, C::kTile);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sK + st * C::kTile + nb * kTileBlockBytes, side ? &mapKs : &mapK, bar_kf + st,
+                      nb * 64, y, kv_plane);
+        if (use > 0) wait(bar_ve + st, (use - 1) & 1);
+        mbar_expect_tx(bar_vf + st, C::kTile);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sV + st * C::kTile + nb * kTileBlockBytes, side ? &mapVs : &mapV, bar_vf + st,
+                      nb * 64, y, kv_plane);
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+      constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+      int n_pv[2] = {0, 0};  // PV MMAs issued per slot
+      bool q_seen[2] = {false, false};
+      for (int s = 0; s <= n_tiles; ++s) {
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const uint32_t tS = tmem + (x ? C::kS1 : C::kS0), tO = tmem + (x ? C::kO1 : C::kO0);
+          if (s >= 1 && active(x, s - 1)) {
+            const int j = s - 1, st = j % NST;
+            wait(bar_p + x, n_pv[x] & 1);
+            wait(bar_vf + st, (j / NST) & 1);
+            tc_fence_after();
+            const uint32_t va = smem_u32(sV + st * C::kTile);
+#pragma unroll
+            for (int k = 0; k < kBN / 16; ++k)
+              umma_ts(tO, tS + k * 8, make_smem_desc(va + k * 2048, kTileBlockBytes, 1024), idesc_o,
+                      (n_pv[x] > 0 || k > 0));
+            ++n_pv[x];
+          }
+          if (s < n_tiles && active(x, s)) {
+            const int st = s % NST;
+            if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
+            wait(bar_kf + st, (s / NST) & 1);
+            tc_fence_after();
+            const uint32_t qa = smem_u32(sQ + x * C::kTile), ka = smem_u32(sK + st * C::kTile);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
+              umma_ss(tS, make_smem_desc(qa + off, 16, 1024), make_smem_desc(ka + off, 16, 1024),
+                      idesc_s, k > 0);
+            }
+            tc_commit(bar_s + x);
+          }
+        }
+        if (s < n_tiles) tc_commit(bar_ke + s % NST);      // every S MMA reading K(s) is issued
+        if (s >= 1) tc_commit(bar_ve + (s - 1) % NST);     // every PV MMA reading V(s-1) is issued
+      }
+      tc_commit(bar_o);
+    }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    // ---------------- softmax of slot x ----------------
+    const int x = (warp >= 8) ? 1 : 0;
+    const int r = tid & 127;                       // row in the tile = tensor-memory lane
+    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_base + (x ? C::kS1 : C::kS0);
+    const uint32_t tO = tmem + lane_base + (x ? C::kO1 : C::kO0);
+    const int t = t_x[x];
+    if (t >= 0) {
+      const int row = t * kBM + r;  // this thread's query position
+      const int q_plane = b * p.Hq + hq_x[x];
+      const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
+      const int side_full = side_full_x[x];
+      float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
+      float l_sum = 0.f;
+      int n_done = 0;
+      uint32_t sreg[4][32];
+      for (int j = 0; j < n_tiles; ++j) {
+        if (!active(x, j)) continue;
+        wait(bar_s + x, n_done & 1);
         tc_fence_after();
-        issue_s(j + 1);
-      }
-    }
-    __syncwarp();
 #pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_ld32(tmem_row + tmem_S0 + st * 128 + c * 32, sreg[c]);
-    tmem_ld_wait();
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, sreg[c]);
+        tmem_ld_wait();
 
-    // kept columns of this tile for this row: [c_lo, c_hi)
-    const bool side = j < n_side_tiles;
-    int c_lo = 0, c_hi = kBN;
-    bool need_mask;
-    if (side) {
-      c_hi = lim_i - j * kBN;
-      need_mask = (j >= side_full);
-    } else {
-      const int key0 = (win_tile_lo + (j - n_side_tiles)) * kBN;
-      c_hi = row - key0 + 1;
-      c_lo = row - p.n_neighbor + 1 - key0;
-      need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-    }
-    float mx = -INFINITY;
-    if (need_mask) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = c * 32 + e;
-          float s = __uint_as_float(sreg[c][e]) * p.scale_log2;
-          s = (col >= c_lo && col < c_hi) ? s : -INFINITY;
-          sreg[c][e] = __float_as_uint(s);
-          mx = fmaxf(mx, s);
+        // kept columns of this tile for this row: [c_lo, c_hi)
+        const bool side = j < ns;
+        int c_lo = 0, c_hi = kBN;
+        bool need_mask;
+        if (side) {
+          c_hi = lim_i - j * kBN;
+          need_mask = (j >= side_full);
+        } else {
+          const int key0 = (wlo + (j - ns)) * kBN;
+          c_hi = row - key0 + 1;
+          c_lo = row - p.n_neighbor + 1 - key0;
+          need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
         }
-    } else {
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (need_mask) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < 4; ++c)
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float s = __uint_as_float(sreg[c][e]) * p.scale_log2;
-          sreg[c][e] = __float_as_uint(s);
-          mx = fmaxf(mx, s);
+            for (int e = 0; e < 32; ++e) {
+              const int col = c * 32 + e;
+              float s = __uint_as_float(sreg[c][e]);
+              s = (col >= c_lo && col < c_hi) ? s : -INFINITY;
+              sreg[c][e] = __float_as_uint(s);
+              mx4[e & 3] = fmaxf(mx4[e & 3], s);
+            }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sreg[c][e]));
         }
-    }
-    // lazy rescale: move the reference only when the maximum grew by more than 2^8
-    float corr = 1.f;
-    bool rescale = false;
-    if (mx > m_ref + 8.f) {
-      corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
-      m_ref = mx;
-      rescale = true;
-    }
-    const float m_eff = (m_ref == -INFINITY) ? 0.f : m_ref;
-    float psum = 0.f;
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+        // lazy rescale: move the reference only when the maximum grew by more than 2^8
+        float corr = 1.f;
+        bool rescale = false;
+        if (mx > m_ref + 8.f) {
+          corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
+          m_ref = mx;
+          rescale = true;
+        }
+        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+        float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 4; ++c)
 #pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float p0 = ex2(__uint_as_float(sreg[c][e]) - m_eff);
-        const float p1 = ex2(__uint_as_float(sreg[c][e + 1]) - m_eff);
-        psum += p0 + p1;
-        sreg[c][e >> 1] = pack_bf16(p0, p1);
-      }
-    l_sum = l_sum * corr + psum;
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sreg[c][e]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sreg[c][e + 1]), p.scale_log2, neg_m));
+            ps4[(e >> 1) & 3] += p0 + p1;
+            sreg[c][e >> 1] = pack_bf16(p0, p1);
+          }
+        l_sum = l_sum * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
 
-    // PV(j-1) must be complete before O is rescaled and before P is overwritten
-    if (j > 0) {
-      wait(bar_o, (j - 1) & 1);
+        // S_x(j) complete means PV_x of the previous tile is complete too: O_x is quiescent
+        if (n_done > 0 && __any_sync(0xffffffffu, rescale)) {
+          uint32_t oreg[32];
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            tmem_ld32(tO + c * 32, oreg);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * corr);
+            tmem_st32(tO + c * 32, oreg);
+          }
+        }
+        // P as packed bf16 over the first 64 columns of S_x: column c holds keys 2c, 2c+1
+        {
+          uint32_t pk[32];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) { pk[e] = sreg[2 * h][e]; pk[16 + e] = sreg[2 * h + 1][e]; }
+            tmem_st32(tS + h * 32, pk);
+          }
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bar_p + x);
+        ++n_done;
+      }
+
+      wait(bar_o, 0);
       tc_fence_after();
-    }
-    __syncwarp();
-    if (leader && j + 1 < n_tiles) load_v(j + 1);  // PV(j-1) is complete, its V stage is free
-    if (j > 0 && __any_sync(0xffffffffu, rescale)) {
-      uint32_t oreg[32];
+      const float inv_l = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      if (row < p.L) p.LSE[size_t(q_plane) * p.L + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+      __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * D;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(tmem_row + tmem_O + c * 32, oreg);
+        uint32_t oreg[32];
+        tmem_ld32(tO + c * 32, oreg);
         tmem_ld_wait();
+        if (row < p.L) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * corr);
-        tmem_st32(tmem_row + tmem_O + c * 32, oreg);
-      }
-      tmem_st_wait();
-    }
-    // P row -> shared memory, bf16, in the swizzled K-major layout the MMA reads
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int chunk16 = c * 4 + q4;  // 16-byte chunk (8 keys) within the row of 128 keys
-        const uint4 val = make_uint4(sreg[c][q4 * 4 + 0], sreg[c][q4 * 4 + 1], sreg[c][q4 * 4 + 2],
-                                     sreg[c][q4 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sP + (chunk16 >> 3) * kTileBlockBytes +
-                                  swz128(tid, chunk16 & 7)) = val;
-      }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (leader) {
-      tc_fence_after();
-      wait(bar_v + st, (j >> 1) & 1);
-      issue_pv(j);
-    }
-  }
-
-  wait(bar_o, (n_tiles - 1) & 1);
-  tc_fence_after();
-  __syncwarp();
-  const float inv_l = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
-  if (row < p.L) p.LSE[size_t(q_plane) * p.L + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-  __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * D;
-#pragma unroll
-  for (int c = 0; c < D / 32; ++c) {
-    uint32_t oreg[32];
-    tmem_ld32(tmem_row + tmem_O + c * 32, oreg);
-    tmem_ld_wait();
-    if (row < p.L) {
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint4 val;
-        val.x = pack_bf16(__uint_as_float(oreg[q4 * 8 + 0]) * inv_l, __uint_as_float(oreg[q4 * 8 + 1]) * inv_l);
-        val.y = pack_bf16(__uint_as_float(oreg[q4 * 8 + 2]) * inv_l, __uint_as_float(oreg[q4 * 8 + 3]) * inv_l);
-        val.z = pack_bf16(__uint_as_float(oreg[q4 * 8 + 4]) * inv_l, __uint_as_float(oreg[q4 * 8 + 5]) * inv_l);
-        val.w = pack_bf16(__uint_as_float(oreg[q4 * 8 + 6]) * inv_l, __uint_as_float(oreg[q4 * 8 + 7]) * inv_l);
-        *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 val;
+            val.x = pack_bf16(__uint_as_float(oreg[q4 * 8 + 0]) * inv_l, __uint_as_float(oreg[q4 * 8 + 1]) * inv_l);
+            val.y = pack_bf16(__uint_as_float(oreg[q4 * 8 + 2]) * inv_l, __uint_as_float(oreg[q4 * 8 + 3]) * inv_l);
+            val.z = pack_bf16(__uint_as_float(oreg[q4 * 8 + 4]) * inv_l, __uint_as_float(oreg[q4 * 8 + 5]) * inv_l);
+            val.w = pack_bf16(__uint_as_float(oreg[q4 * 8 + 6]) * inv_l, __uint_as_float(oreg[q4 * 8 + 7]) * inv_l);
+            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
+          }
+        }
       }
     }
   }
@@ -460,12 +519,16 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.n_neighbor = id->n_neighbor;
   p.side_cap = id->side_cap;
   p.side_tiles_cap = lay.cap_pad / 128;
+  const int G = d->Hq / d->Hkv;
+  p.pair_heads = (G % 2 == 0) ? 1 : 0;
   const float scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
   p.scale_log2 = scale * 1.4426950408889634f;
-  const uint32_t smem = FwdSmem<D>::kRequest;
+  const uint32_t smem = FwdCfg<D>::kRequest;
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_kernel<D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-  attn_fwd_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), 128, smem, stream>>>(mq, mk, mv, mks, mvs, p);
+  const dim3 grid = p.pair_heads ? dim3(ih.n_tiles, d->Hq / 2, d->B)
+                                 : dim3((ih.n_tiles + 1) / 2, d->Hq, d->B);
+  attn_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, mks, mvs, p);
   record_event(d, 2, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;

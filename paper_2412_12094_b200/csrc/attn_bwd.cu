@@ -20,12 +20,12 @@ namespace sepllm {
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ---------------------------------------------------------------------------
-// Delta
+// Row statistics: (LSE in log2 units, Delta) per query row
 // ---------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_delta(const __nv_bfloat16* __restrict__ dO, const __nv_bfloat16* __restrict__ O,
-          float* __restrict__ delta, size_t rows) {
+          const float* __restrict__ LSE, float2* __restrict__ stats, size_t rows) {
   constexpr int LPR = D / 8;
   const size_t r = (size_t(blockIdx.x) * 256 + threadIdx.x) / LPR;
   const int l = threadIdx.x % LPR;
@@ -44,7 +44,7 @@ bwd_delta(const __nv_bfloat16* __restrict__ dO, const __nv_bfloat16* __restrict_
   }
 #pragma unroll
   for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if (r < rows && l == 0) delta[r] = s;
+  if (r < rows && l == 0) stats[r] = make_float2(LSE[r] * kLog2e, s);
 }
 
 struct BwdParams {
@@ -53,15 +53,14 @@ struct BwdParams {
   const int32_t* side_pos;   // [B][side_cap]
   const int32_t* n_side;     // [B]
   const int32_t* tile_meta;  // [B][T][8]
-  const float* LSE;          // [B][Hq][L]
-  const float* delta;        // [B][Hq][L]
-  float* dKs;                // [B][Hkv][cap_pad][D] fp32 side partials
+  const float2* stats;       // [B][Hq][L] (LSE * log2 e, Delta)
+  float* dKs;                // [split][B][Hkv][cap_pad][D] fp32 side partials
   float* dVs;
   void* dQ;
   void* dK;
   void* dV;
   int32_t* status;
-  int L, T, Hq, Hkv, n_neighbor, side_cap, cap_pad, grad_fp32;
+  int L, T, Hq, Hkv, n_neighbor, side_cap, cap_pad, grad_fp32, split, pair_heads;
   float scale, scale_log2;
 };
 
@@ -80,60 +79,111 @@ __device__ __forceinline__ void store_row_chunk32(void* base, size_t elem_off, i
   }
 }
 
+constexpr int kBwdThreads = 384;
+constexpr uint32_t kHalfBlockBytes = 64 * 128;  // 64 rows x 64 bf16, one swizzled block
+constexpr int kFar = 0x3fffffff;                // "never" / "unbounded" for column ranges
+
 // ---------------------------------------------------------------------------
 // dQ: query-tile stationary
 // ---------------------------------------------------------------------------
+// Same shape as the forward: two query-tile slots per CTA sharing their key tiles, a TMA warp, an
+// MMA warp and one arithmetic warpgroup per slot.  Keys are taken 64 at a time so that a slot's
+// S, dP (64 columns each) and dQ (D columns) fit in half of tensor memory:
+//   S_x = Q_x K_h^T, dP_x = dO_x V_h^T  ->  dS = P (dP - Delta) written as packed bf16 over S_x
+//   dQ_x += dS K_h  (A operand from tensor memory).
 template <int D>
-struct DqSmem {
+struct DqCfg {
   static constexpr int NB = D / 64;
-  static constexpr uint32_t kQ = 0;
-  static constexpr uint32_t kdO = kQ + NB * kTileBlockBytes;
-  static constexpr uint32_t kK = kdO + NB * kTileBlockBytes;
-  static constexpr uint32_t kV = kK + 2 * NB * kTileBlockBytes;
-  static constexpr uint32_t kdS = kV + 2 * NB * kTileBlockBytes;
-  static constexpr uint32_t kBar = kdS + 2 * kTileBlockBytes;
-  static constexpr uint32_t kTotal = kBar + 256;
+  static constexpr int NSK = 3, NSV = 2;            // K_h is read by two consecutive steps
+  static constexpr uint32_t kTile = NB * kTileBlockBytes;
+  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;
+  static constexpr uint32_t kQ = 0;                 // Q_0, Q_1
+  static constexpr uint32_t kdO = kQ + 2 * kTile;   // dO_0, dO_1
+  static constexpr uint32_t kK = kdO + 2 * kTile;
+  static constexpr uint32_t kV = kK + NSK * kHalf;
+  static constexpr uint32_t kBar = kV + NSV * kHalf;
+  static constexpr uint32_t kTotal = kBar + 512;
   static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
+  // tensor-memory columns: per slot S (64) | dP (64) | dQ (D)
+  static constexpr uint32_t kSlot = 256, kS = 0, kdP = 64, kdQ = 128;
 };
 
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
               const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
               const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
               const BwdParams p) {
-  using SM = DqSmem<D>;
-  constexpr int NB = SM::NB;
+  using C = DqCfg<D>;
+  constexpr int NB = C::NB, NSK = C::NSK, NSV = C::NSV;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* sQ = smem + SM::kQ;
-  uint8_t* sdO = smem + SM::kdO;
-  uint8_t* sK = smem + SM::kK;
-  uint8_t* sV = smem + SM::kV;
-  uint8_t* sdS = smem + SM::kdS;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBar);
-  uint64_t* bar_q = bars + 0;
-  uint64_t* bar_k = bars + 1;   // [2]
-  uint64_t* bar_v = bars + 3;   // [2]
-  uint64_t* bar_sp = bars + 5;  // S and dP of a tile are complete
-  uint64_t* bar_dq = bars + 6;  // dQ MMA of a tile is complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+  uint8_t* sQ = smem + C::kQ;
+  uint8_t* sdO = smem + C::kdO;
+  uint8_t* sK = smem + C::kK;
+  uint8_t* sV = smem + C::kV;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
+  uint64_t* bar_q = bars;              // [2]   Q_x and dO_x landed
+  uint64_t* bar_sp = bars + 2;         // [2]   S_x and dP_x complete
+  uint64_t* bar_ds = bars + 4;         // [2]   dS_x written by its 128 threads
+  uint64_t* bar_acc = bars + 6;        //       every MMA complete
+  uint64_t* bar_kf = bars + 8;         // [NSK]
+  uint64_t* bar_ke = bar_kf + NSK;     // [NSK]
+  uint64_t* bar_vf = bar_ke + NSK;     // [NSV]
+  uint64_t* bar_ve = bar_vf + NSV;     // [NSV]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + 2 * NSK + 2 * NSV);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const bool leader = (tid == 0);
-  const int t = p.T - 1 - int(blockIdx.x);
-  const int hq = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
-  const int q_plane = b * p.Hq + hq;
-  const int kv_plane = b * p.Hkv + hq / G;
+  int t_x[2], hq_x[2];
+  if (p.pair_heads) {
+    t_x[0] = t_x[1] = p.T - 1 - int(blockIdx.x);
+    hq_x[0] = 2 * int(blockIdx.y);
+    hq_x[1] = hq_x[0] + 1;
+  } else {
+    t_x[1] = p.T - 1 - 2 * int(blockIdx.x);
+    t_x[0] = t_x[1] - 1;
+    hq_x[0] = hq_x[1] = int(blockIdx.y);
+  }
+  const int kv_plane = b * p.Hkv + hq_x[0] / G;
+  int side_full_x[2], ns_x[2], wlo_x[2], whi_x[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    if (t_x[x] >= 0) {
+      const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t_x[x]) * 8;
+      side_full_x[x] = meta[0];
+      ns_x[x] = min(meta[1], p.cap_pad / kBN);
+      wlo_x[x] = meta[4];
+      whi_x[x] = meta[5];
+    } else {
+      side_full_x[x] = 0; ns_x[x] = 0; wlo_x[x] = 0; whi_x[x] = 0;
+    }
+  }
+  if (t_x[0] < 0) { wlo_x[0] = wlo_x[1]; whi_x[0] = wlo_x[1]; }
+  const int ns = max(ns_x[0], ns_x[1]);
+  const int wlo = min(wlo_x[0], wlo_x[1]);
+  const int whi = max(whi_x[0], whi_x[1]);
+  const int n_steps = 2 * (ns + (whi - wlo));  // key half-tiles
+  auto active = [&](int x, int s) -> bool {
+    const int j = s >> 1;
+    if (j < ns) return j < ns_x[x];
+    const int w = wlo + (j - ns);
+    return w >= wlo_x[x] && w < whi_x[x];
+  };
+  // first key row of half-tile s in its tensor (side buffer or K/V)
+  auto half_y = [&](int s) -> int {
+    const int j = s >> 1;
+    return ((j < ns) ? j * kBN : (wlo + (j - ns)) * kBN) + (s & 1) * 64;
+  };
 
-  if (leader) {
-    mbar_init(bar_q, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_k + i, 1); mbar_init(bar_v + i, 1); }
-    mbar_init(bar_sp, 1);
-    mbar_init(bar_dq, 1);
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 128); }
+    mbar_init(bar_acc, 1);
+    for (int i = 0; i < NSK; ++i) { mbar_init(bar_kf + i, 1); mbar_init(bar_ke + i, 1); }
+    for (int i = 0; i < NSV; ++i) { mbar_init(bar_vf + i, 1); mbar_init(bar_ve + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -146,37 +196,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_row = tmem + (uint32_t(warp * 32) << 16);
-  constexpr uint32_t tmem_S = 0, tmem_dP = 128, tmem_dQ = 256;
 
-  const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t) * 8;
-  const int side_full = meta[0];
-  const int n_side_tiles = min(meta[1], p.cap_pad / kBN);
-  const int win_tile_lo = meta[4];
-  const int n_tiles = n_side_tiles + (meta[5] - win_tile_lo);
-  const int row = t * kBM + tid;
-  const bool row_ok = row < p.L;
-  const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-  const float lse2 = row_ok ? p.LSE[size_t(q_plane) * p.L + row] * kLog2e : INFINITY;
-  const float delta_i = row_ok ? p.delta[size_t(q_plane) * p.L + row] : 0.f;
-
-  auto tile_y = [&](int j) {
-    return (j < n_side_tiles) ? j * kBN : (win_tile_lo + (j - n_side_tiles)) * kBN;
-  };
-  auto load_k = [&](int j) {
-    const int st = j & 1;
-    mbar_expect_tx(bar_k + st, NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb)
-      tma_load_3d(sK + (st * NB + nb) * kTileBlockBytes, (j < n_side_tiles) ? &mapKs : &mapK,
-                  bar_k + st, nb * 64, tile_y(j), kv_plane);
-  };
-  auto load_v = [&](int j) {
-    const int st = j & 1;
-    mbar_expect_tx(bar_v + st, NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb)
-      tma_load_3d(sV + (st * NB + nb) * kTileBlockBytes, (j < n_side_tiles) ? &mapVs : &mapV,
-                  bar_v + st, nb * 64, tile_y(j), kv_plane);
-  };
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (!mbar_wait(bar, parity, abort_flag)) {
@@ -184,125 +204,161 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       ok = false;
     }
   };
-  constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
-  constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
 
-  if (leader) {
-    mbar_expect_tx(bar_q, 2 * NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb) {
-      tma_load_3d(sQ + nb * kTileBlockBytes, &mapQ, bar_q, nb * 64, t * kBM, q_plane);
-      tma_load_3d(sdO + nb * kTileBlockBytes, &mapdO, bar_q, nb * 64, t * kBM, q_plane);
-    }
-    load_k(0);
-    load_v(0);
-    if (n_tiles > 1) { load_k(1); load_v(1); }
-    wait(bar_q, 0);
-  }
-
-  for (int j = 0; j < n_tiles; ++j) {
-    const int st = j & 1;
-    if (leader) {
-      const uint32_t qa = smem_u32(sQ), doa = smem_u32(sdO);
-      const uint32_t ka = smem_u32(sK + st * NB * kTileBlockBytes);
-      const uint32_t va = smem_u32(sV + st * NB * kTileBlockBytes);
-      wait(bar_k + st, (j >> 1) & 1);
-      tc_fence_after();
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 0 && lane == 0) {
+      // ---------------- TMA producer ----------------
 #pragma unroll
-      for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_S, make_smem_desc(qa + off, 16, 1024), make_smem_desc(ka + off, 16, 1024),
-                idesc_s, k > 0);
-      }
-      wait(bar_v + st, (j >> 1) & 1);
-      tc_fence_after();
-#pragma unroll
-      for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_dP, make_smem_desc(doa + off, 16, 1024),
-                make_smem_desc(va + off, 16, 1024), idesc_s, k > 0);
-      }
-      tc_commit(bar_sp);
-    }
-    wait(bar_sp, j & 1);
-    tc_fence_after();
-    if (leader && j + 2 < n_tiles) load_v(j + 2);  // dP(j) is complete: its V stage is free
-    __syncwarp();
-
-    const bool side = j < n_side_tiles;
-    int c_lo = 0, c_hi = kBN;
-    bool need_mask;
-    if (side) {
-      c_hi = lim_i - j * kBN;
-      need_mask = (j >= side_full);
-    } else {
-      const int key0 = tile_y(j);
-      c_hi = row - key0 + 1;
-      c_lo = row - p.n_neighbor + 1 - key0;
-      need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-    }
-    // dQ MMA of the previous tile reads sdS and its K stage
-    if (j > 0) {
-      wait(bar_dq, (j - 1) & 1);
-      tc_fence_after();
-      if (leader && j + 1 < n_tiles && j >= 1) {
-        if (j + 1 >= 2) load_k(j + 1);  // K stage of tile j-1 is free now
-      }
-    }
-    __syncwarp();
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t s[32], dp[32];
-      tmem_ld32(tmem_row + tmem_S + c * 32, s);
-      tmem_ld32(tmem_row + tmem_dP + c * 32, dp);
-      tmem_ld_wait();
-#pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        float ds[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int col = c * 32 + e + u;
-          float pr = ex2(__uint_as_float(s[e + u]) * p.scale_log2 - lse2);
-          if (need_mask && !(col >= c_lo && col < c_hi)) pr = 0.f;
-          ds[u] = pr * (__uint_as_float(dp[e + u]) - delta_i);
+      for (int x = 0; x < 2; ++x)
+        if (t_x[x] >= 0) {
+          mbar_expect_tx(bar_q + x, 2 * C::kTile);
+          for (int nb = 0; nb < NB; ++nb) {
+            tma_load_3d(sQ + x * C::kTile + nb * kTileBlockBytes, &mapQ, bar_q + x, nb * 64,
+                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+            tma_load_3d(sdO + x * C::kTile + nb * kTileBlockBytes, &mapdO, bar_q + x, nb * 64,
+                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+          }
         }
-        s[e >> 1] = pack_bf16(ds[0], ds[1]);
+      for (int s = 0; s < n_steps; ++s) {
+        const bool side = (s >> 1) < ns;
+        const int y = half_y(s);
+        const int sk = s % NSK, sv = s % NSV;
+        if (s >= NSK) wait(bar_ke + sk, (s / NSK - 1) & 1);
+        mbar_expect_tx(bar_kf + sk, C::kHalf);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sK + sk * C::kHalf + nb * kHalfBlockBytes, side ? &mapKs : &mapK, bar_kf + sk,
+                      nb * 64, y, kv_plane);
+        if (s >= NSV) wait(bar_ve + sv, (s / NSV - 1) & 1);
+        mbar_expect_tx(bar_vf + sv, C::kHalf);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sV + sv * C::kHalf + nb * kHalfBlockBytes, side ? &mapVs : &mapV, bar_vf + sv,
+                      nb * 64, y, kv_plane);
       }
+    } else if (warp == 1 && lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
+      int n_dq[2] = {0, 0};
+      bool q_seen[2] = {false, false};
+      for (int s = 0; s <= n_steps; ++s) {
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int chunk16 = c * 4 + q4;
-        *reinterpret_cast<uint4*>(sdS + (chunk16 >> 3) * kTileBlockBytes + swz128(tid, chunk16 & 7)) =
-            make_uint4(s[q4 * 4], s[q4 * 4 + 1], s[q4 * 4 + 2], s[q4 * 4 + 3]);
+        for (int x = 0; x < 2; ++x) {
+          const uint32_t tb = tmem + x * C::kSlot;
+          if (s >= 1 && active(x, s - 1)) {
+            const int sk = (s - 1) % NSK;
+            wait(bar_ds + x, n_dq[x] & 1);
+            tc_fence_after();
+            const uint32_t ka = smem_u32(sK + sk * C::kHalf);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_ts(tb + C::kdQ, tb + C::kS + k * 8,
+                      make_smem_desc(ka + k * 2048, kHalfBlockBytes, 1024), idesc_dq,
+                      (n_dq[x] > 0 || k > 0));
+            ++n_dq[x];
+          }
+          if (s < n_steps && active(x, s)) {
+            const int sk = s % NSK, sv = s % NSV;
+            if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
+            wait(bar_kf + sk, (s / NSK) & 1);
+            tc_fence_after();
+            const uint32_t qa = smem_u32(sQ + x * C::kTile), doa = smem_u32(sdO + x * C::kTile);
+            const uint32_t ka = smem_u32(sK + sk * C::kHalf), va = smem_u32(sV + sv * C::kHalf);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k)
+              umma_ss(tb + C::kS,
+                      make_smem_desc(qa + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
+                      make_smem_desc(ka + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024),
+                      idesc_s, k > 0);
+            wait(bar_vf + sv, (s / NSV) & 1);
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k)
+              umma_ss(tb + C::kdP,
+                      make_smem_desc(doa + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
+                      make_smem_desc(va + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024),
+                      idesc_s, k > 0);
+            tc_commit(bar_sp + x);
+          }
+        }
+        if (s < n_steps) tc_commit(bar_ve + s % NSV);       // dP MMAs reading V_h(s) are issued
+        if (s >= 1) tc_commit(bar_ke + (s - 1) % NSK);      // S(s-1) and dQ(s-1) MMAs are issued
       }
+      tc_commit(bar_acc);
     }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (leader) {
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    // ---------------- dS of slot x ----------------
+    const int x = (warp >= 8) ? 1 : 0;
+    const int r = tid & 127;
+    const uint32_t tb = tmem + (uint32_t((warp & 3) * 32) << 16) + x * C::kSlot;
+    const int t = t_x[x];
+    if (t >= 0) {
+      const int row = t * kBM + r;
+      const bool row_ok = row < p.L;
+      const int q_plane = b * p.Hq + hq_x[x];
+      const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
+      const float2 st = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
+      const float neg_lse2 = -st.x, delta_i = st.y;
+      const int side_full = side_full_x[x];
+      int n_done = 0;
+      for (int s = 0; s < n_steps; ++s) {
+        if (!active(x, s)) continue;
+        const int j = s >> 1;
+        const bool side = j < ns;
+        int c_lo = 0, c_hi = 64;
+        bool need_mask;
+        if (side) {
+          c_hi = lim_i - half_y(s);
+          need_mask = (j >= side_full);
+        } else {
+          const int key0 = half_y(s);
+          c_hi = row - key0 + 1;
+          c_lo = row - p.n_neighbor + 1 - key0;
+          need_mask = (key0 + 63 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
+        }
+        wait(bar_sp + x, n_done & 1);
+        tc_fence_after();
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sv[32], dp[32];
+          tmem_ld32(tb + C::kS + c * 32, sv);
+          tmem_ld32(tb + C::kdP + c * 32, dp);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float ds[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int col = c * 32 + e + u;
+              float pr = ex2(fmaf(__uint_as_float(sv[e + u]), p.scale_log2, neg_lse2));
+              if (need_mask && !(col >= c_lo && col < c_hi)) pr = 0.f;
+              ds[u] = pr * (__uint_as_float(dp[e + u]) - delta_i);
+            }
+            pk[c * 16 + (e >> 1)] = pack_bf16(ds[0], ds[1]);
+          }
+        }
+        tmem_st32(tb + C::kS, pk);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bar_ds + x);
+        ++n_done;
+      }
+      wait(bar_acc, 0);
       tc_fence_after();
-      const uint32_t dsa = smem_u32(sdS), ka = smem_u32(sK + st * NB * kTileBlockBytes);
 #pragma unroll
-      for (int k = 0; k < kBN / 16; ++k) {
-        const uint32_t aoff = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_dQ, make_smem_desc(dsa + aoff, 16, 1024),
-                make_smem_desc(ka + k * 2048, kTileBlockBytes, 1024), idesc_dq, (j > 0 || k > 0));
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t rr[32];
+        tmem_ld32(tb + C::kdQ + c * 32, rr);
+        tmem_ld_wait();
+        if (row_ok) {
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
+          store_row_chunk32(p.dQ, (size_t(q_plane) * p.L + row) * D + c * 32, p.grad_fp32, v);
+        }
       }
-      tc_commit(bar_dq);
-    }
-  }
-
-  wait(bar_dq, (n_tiles - 1) & 1);
-  tc_fence_after();
-  __syncwarp();
-#pragma unroll
-  for (int c = 0; c < D / 32; ++c) {
-    uint32_t r[32];
-    tmem_ld32(tmem_row + tmem_dQ + c * 32, r);
-    tmem_ld_wait();
-    if (row_ok) {
-      float v[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * p.scale;
-      store_row_chunk32(p.dQ, (size_t(q_plane) * p.L + row) * D + c * 32, p.grad_fp32, v);
     }
   }
   tc_fence_before();
@@ -313,74 +369,86 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 // ---------------------------------------------------------------------------
 // dK, dV: key-tile stationary
 // ---------------------------------------------------------------------------
+// One CTA owns 128 keys and streams the query rows that keep any of them, 64 rows of one query
+// head at a time ("half-iteration"), through a ring of NSTQ stages:
+//   warp 0      TMA producer (K, V once; then Q_h, dO_h per half-iteration)
+//   warp 1      MMA issuer:  S^T = K Q_h^T and dP^T = V dO_h^T into one of two tensor-memory
+//               buffers; later dV += P^T dO_h and dK += dS^T Q_h with A taken from tensor memory
+//   warps 2-3   load the 64 (LSE, Delta) pairs of the half-iteration into shared memory
+//   warps 4-7   P^T, dS^T of even half-iterations (thread = key row), written as packed bf16
+//               over the S^T / dP^T columns they came from
+//   warps 8-11  the same for odd half-iterations
 template <int D>
-struct DkvSmem {
+struct DkvCfg {
   static constexpr int NB = D / 64;
+  static constexpr int NSTQ = 4;
+  static constexpr uint32_t kTile = NB * kTileBlockBytes;
+  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;
   static constexpr uint32_t kK = 0;
-  static constexpr uint32_t kV = kK + NB * kTileBlockBytes;
-  static constexpr uint32_t kQ = kV + NB * kTileBlockBytes;
-  static constexpr uint32_t kdO = kQ + NB * kTileBlockBytes;
-  static constexpr uint32_t kPT = kdO + NB * kTileBlockBytes;
-  static constexpr uint32_t kdST = kPT + 2 * kTileBlockBytes;
-  static constexpr uint32_t kRow = kdST + 2 * kTileBlockBytes;  // lse2[128], delta[128], lim[128]
-  static constexpr uint32_t kBar = kRow + 3 * 128 * 4;
-  static constexpr uint32_t kTotal = kBar + 256;
+  static constexpr uint32_t kV = kK + kTile;
+  static constexpr uint32_t kQ = kV + kTile;                 // NSTQ x [Q_h | dO_h]
+  static constexpr uint32_t kStat = kQ + NSTQ * 2 * kHalf;   // NSTQ x 64 float2
+  static constexpr uint32_t kBar = kStat + NSTQ * 64 * 8;
+  static constexpr uint32_t kTotal = kBar + 512;
   static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
+  // tensor-memory columns
+  static constexpr uint32_t kdV = 0, kdK = D, kBuf = 256, kBufStride = 128, kST = 0, kdPT = 64;
 };
 
 template <int D, bool SIDE>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
                const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const BwdParams p) {
-  using SM = DkvSmem<D>;
-  constexpr int NB = SM::NB;
+  using C = DkvCfg<D>;
+  constexpr int NB = C::NB, NSTQ = C::NSTQ;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* sK = smem + SM::kK;
-  uint8_t* sV = smem + SM::kV;
-  uint8_t* sQ = smem + SM::kQ;
-  uint8_t* sdO = smem + SM::kdO;
-  uint8_t* sPT = smem + SM::kPT;
-  uint8_t* sdST = smem + SM::kdST;
-  float* s_lse2 = reinterpret_cast<float*>(smem + SM::kRow);
-  float* s_delta = s_lse2 + 128;
-  int32_t* s_lim = reinterpret_cast<int32_t*>(s_delta + 128);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBar);
-  uint64_t* bar_kv = bars + 0;
-  uint64_t* bar_qdo = bars + 1;
-  uint64_t* bar_sp = bars + 2;
-  uint64_t* bar_acc = bars + 3;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+  uint8_t* sK = smem + C::kK;
+  uint8_t* sV = smem + C::kV;
+  uint8_t* sQ = smem + C::kQ;
+  float2* s_stat = reinterpret_cast<float2*>(smem + C::kStat);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
+  uint64_t* bar_kv = bars;              //        K, V landed
+  uint64_t* bar_acc = bars + 1;         //        every MMA complete
+  uint64_t* bar_sp = bars + 2;          // [2]    S^T and dP^T of buffer u complete
+  uint64_t* bar_pds = bars + 4;         // [2]    P^T and dS^T of buffer u written
+  uint64_t* bar_qf = bars + 6;          // [NSTQ] Q_h, dO_h landed
+  uint64_t* bar_qe = bar_qf + NSTQ;     // [NSTQ] stage free (its dV / dK MMAs are complete)
+  uint64_t* bar_sf = bar_qe + NSTQ;     // [NSTQ] row statistics written
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 3 * NSTQ);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const bool leader = (tid == 0);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kt = SIDE ? int(blockIdx.x) : int(gridDim.x) - 1 - int(blockIdx.x);
-  const int hk = blockIdx.y, b = blockIdx.z;
+  const int b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
+  // the side pass may give each query head of the group its own CTA (and partial buffer)
+  const int split = SIDE ? p.split : 1;
+  const int hk = int(blockIdx.y) / split, part = int(blockIdx.y) % split;
+  const int g_lo = (split > 1) ? part : 0, n_g = (split > 1) ? 1 : G;
   const int kv_plane = b * p.Hkv + hk;
   const int ns = min(p.n_side[b], p.side_cap);
+  const int QH = (p.L + 63) / 64;
 
-  // query tiles that keep at least one key of this tile
-  int t_lo, t_hi;
+  // query half-tiles [qh_lo, qh_hi] that keep at least one key of this tile
+  int qh_lo, qh_hi;
   if (SIDE) {
     if (kt * kBN >= ns) return;  // no entries in this side tile: nothing reads its partial rows
-    t_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / kBM;
-    t_hi = p.T - 1;
+    qh_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / 64;
+    qh_hi = QH - 1;
   } else {
-    t_lo = kt;  // kBM == kBN
-    t_hi = min(p.T - 1, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / kBM);
+    qh_lo = 2 * kt;  // kBM == kBN
+    qh_hi = min(QH - 1, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / 64);
   }
-  const int n_qt = max(0, t_hi - t_lo + 1);
-  const int n_iter = n_qt * G;
+  const int n_it = max(0, qh_hi - qh_lo + 1) * n_g;
 
-  if (leader) {
+  if (tid == 0) {
     mbar_init(bar_kv, 1);
-    mbar_init(bar_qdo, 1);
-    mbar_init(bar_sp, 1);
     mbar_init(bar_acc, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_pds + i, 128); }
+    for (int i = 0; i < NSTQ; ++i) { mbar_init(bar_qf + i, 1); mbar_init(bar_qe + i, 1); mbar_init(bar_sf + i, 64); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -393,8 +461,6 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_row = tmem + (uint32_t(warp * 32) << 16);
-  constexpr uint32_t tmem_ST = 0, tmem_dPT = 128, tmem_dV = 256, tmem_dK = 256 + D;
 
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
@@ -403,205 +469,215 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       ok = false;
     }
   };
-  auto load_qdo = [&](int it) {
-    const int tq = t_lo + it / G, g = it % G;
-    const int q_plane = b * p.Hq + hk * G + g;
-    mbar_expect_tx(bar_qdo, 2 * NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb) {
-      tma_load_3d(sQ + nb * kTileBlockBytes, &mapQ, bar_qdo, nb * 64, tq * kBM, q_plane);
-      tma_load_3d(sdO + nb * kTileBlockBytes, &mapdO, bar_qdo, nb * 64, tq * kBM, q_plane);
-    }
-  };
-  constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
-  constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);
+  auto q_plane_of = [&](int it) { return b * p.Hq + hk * G + g_lo + it % n_g; };
+  auto q0_of = [&](int it) { return (qh_lo + it / n_g) * 64; };
 
-  if (leader && n_iter > 0) {
-    mbar_expect_tx(bar_kv, 2 * NB * kTileBlockBytes);
-    for (int nb = 0; nb < NB; ++nb) {
-      tma_load_3d(sK + nb * kTileBlockBytes, &mapK, bar_kv, nb * 64, kt * kBN, kv_plane);
-      tma_load_3d(sV + nb * kTileBlockBytes, &mapV, bar_kv, nb * 64, kt * kBN, kv_plane);
-    }
-    load_qdo(0);
-    wait(bar_kv, 0);
-  }
-
-  const int key = kt * kBN + tid;  // side entry index (SIDE) or key position (window)
-
-  for (int it = 0; it < n_iter; ++it) {
-    const int tq = t_lo + it / G, g = it % G;
-    const int q_plane = b * p.Hq + hk * G + g;
-    if (it > 0) {
-      // dV/dK MMAs of the previous iteration read sQ, sdO, sPT, sdST
-      wait(bar_acc, (it - 1) & 1);
-      tc_fence_after();
-      if (leader) load_qdo(it);
-    }
-    __syncthreads();  // previous readers of the per-row arrays are done
-    {
-      const int qi = tq * kBM + tid;
-      const bool q_ok = qi < p.L;
-      s_lse2[tid] = q_ok ? p.LSE[size_t(q_plane) * p.L + qi] * kLog2e : INFINITY;
-      s_delta[tid] = q_ok ? p.delta[size_t(q_plane) * p.L + qi] : 0.f;
-      if (SIDE) s_lim[tid] = q_ok ? min(p.lim[size_t(b) * p.L + qi], p.side_cap) : 0x7fffffff;
-    }
-    if (leader) {
-      wait(bar_qdo, it & 1);
-      tc_fence_after();
-      const uint32_t ka = smem_u32(sK), va = smem_u32(sV), qa = smem_u32(sQ), doa = smem_u32(sdO);
-#pragma unroll
-      for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_ST, make_smem_desc(ka + off, 16, 1024), make_smem_desc(qa + off, 16, 1024),
-                idesc_s, k > 0);
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 0 && lane == 0 && n_it > 0) {
+      // ---------------- TMA producer ----------------
+      mbar_expect_tx(bar_kv, 2 * C::kTile);
+      for (int nb = 0; nb < NB; ++nb) {
+        tma_load_3d(sK + nb * kTileBlockBytes, &mapK, bar_kv, nb * 64, kt * kBN, kv_plane);
+        tma_load_3d(sV + nb * kTileBlockBytes, &mapV, bar_kv, nb * 64, kt * kBN, kv_plane);
       }
-#pragma unroll
-      for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_dPT, make_smem_desc(va + off, 16, 1024),
-                make_smem_desc(doa + off, 16, 1024), idesc_s, k > 0);
-      }
-      tc_commit(bar_sp);
-    }
-    __syncthreads();  // per-row arrays are written
-
-    // kept query columns for this key row: [q_lo, q_hi)
-    int q_lo, q_hi = kBM;
-    bool need_mask;
-    if (SIDE) {
-      // lim is non-decreasing: kept from the first query with lim > key
-      int lo = 0, hi = kBM;
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (s_lim[mid] > key) hi = mid; else lo = mid + 1;
-      }
-      q_lo = lo;
-      need_mask = true;
-    } else {
-      q_lo = key - tq * kBM;
-      q_hi = key + p.n_neighbor - tq * kBM;
-      need_mask = true;
-    }
-    wait(bar_sp, it & 1);
-    tc_fence_after();
-    __syncwarp();
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t s[32], dp[32];
-      tmem_ld32(tmem_row + tmem_ST + c * 32, s);
-      tmem_ld32(tmem_row + tmem_dPT + c * 32, dp);
-      tmem_ld_wait();
-#pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        float pr[2], ds[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int col = c * 32 + e + u;
-          pr[u] = ex2(__uint_as_float(s[e + u]) * p.scale_log2 - s_lse2[col]);
-          if (need_mask && !(col >= q_lo && col < q_hi)) pr[u] = 0.f;
-          ds[u] = pr[u] * (__uint_as_float(dp[e + u]) - s_delta[col]);
+      for (int it = 0; it < n_it; ++it) {
+        const int st = it % NSTQ;
+        if (it >= NSTQ) wait(bar_qe + st, (it / NSTQ - 1) & 1);
+        mbar_expect_tx(bar_qf + st, 2 * C::kHalf);
+        uint8_t* dq = sQ + st * 2 * C::kHalf;
+        const int y = q0_of(it), plane = q_plane_of(it);
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_3d(dq + nb * kHalfBlockBytes, &mapQ, bar_qf + st, nb * 64, y, plane);
+          tma_load_3d(dq + C::kHalf + nb * kHalfBlockBytes, &mapdO, bar_qf + st, nb * 64, y, plane);
         }
-        s[e >> 1] = pack_bf16(pr[0], pr[1]);
-        dp[e >> 1] = pack_bf16(ds[0], ds[1]);
       }
+    } else if (warp == 1 && lane == 0 && n_it > 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t ka = smem_u32(sK), va = smem_u32(sV);
+      auto issue_sp = [&](int it) {
+        const int st = it % NSTQ, u = it & 1;
+        wait(bar_qf + st, (it / NSTQ) & 1);
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sQ + st * 2 * C::kHalf), doa = qa + C::kHalf;
+        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int chunk16 = c * 4 + q4;
-        const uint32_t off = (chunk16 >> 3) * kTileBlockBytes + swz128(tid, chunk16 & 7);
-        *reinterpret_cast<uint4*>(sPT + off) = make_uint4(s[q4 * 4], s[q4 * 4 + 1], s[q4 * 4 + 2], s[q4 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sdST + off) = make_uint4(dp[q4 * 4], dp[q4 * 4 + 1], dp[q4 * 4 + 2], dp[q4 * 4 + 3]);
-      }
-    }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (leader) {
-      tc_fence_after();
-      const uint32_t pta = smem_u32(sPT), dsta = smem_u32(sdST), qa = smem_u32(sQ), doa = smem_u32(sdO);
+        for (int k = 0; k < D / 16; ++k)
+          umma_ss(tb + C::kST,
+                  make_smem_desc(ka + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
+                  make_smem_desc(qa + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024), idesc_s,
+                  k > 0);
 #pragma unroll
-      for (int k = 0; k < kBM / 16; ++k) {
-        const uint32_t aoff = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_dV, make_smem_desc(pta + aoff, 16, 1024),
-                make_smem_desc(doa + k * 2048, kTileBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
-      }
+        for (int k = 0; k < D / 16; ++k)
+          umma_ss(tb + C::kdPT,
+                  make_smem_desc(va + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
+                  make_smem_desc(doa + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024), idesc_s,
+                  k > 0);
+        tc_commit(bar_sp + u);
+      };
+      wait(bar_kv, 0);
+      issue_sp(0);
+      if (n_it > 1) issue_sp(1);
+      for (int it = 0; it < n_it; ++it) {
+        const int st = it % NSTQ, u = it & 1;
+        wait(bar_pds + u, (it >> 1) & 1);
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sQ + st * 2 * C::kHalf), doa = qa + C::kHalf;
+        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
 #pragma unroll
-      for (int k = 0; k < kBM / 16; ++k) {
-        const uint32_t aoff = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-        umma_ss(tmem + tmem_dK, make_smem_desc(dsta + aoff, 16, 1024),
-                make_smem_desc(qa + k * 2048, kTileBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
+        for (int k = 0; k < 4; ++k)
+          umma_ts(tmem + C::kdV, tb + C::kST + k * 8,
+                  make_smem_desc(doa + k * 2048, kHalfBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_ts(tmem + C::kdK, tb + C::kdPT + k * 8,
+                  make_smem_desc(qa + k * 2048, kHalfBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
+        tc_commit(bar_qe + st);
+        if (it + 2 < n_it) issue_sp(it + 2);
       }
       tc_commit(bar_acc);
-    }
-  }
-
-  if (n_iter > 0) {
-    wait(bar_acc, (n_iter - 1) & 1);
-    tc_fence_after();
-  }
-  __syncwarp();
-
-  if (SIDE) {
-    // fp32 partial rows for the entries of this side tile
-    const bool r_ok = key < p.cap_pad;
-    float* dks = p.dKs + (size_t(kv_plane) * p.cap_pad + key) * D;
-    float* dvs = p.dVs + (size_t(kv_plane) * p.cap_pad + key) * D;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t rk[32], rv[32];
-      if (n_iter > 0) {
-        tmem_ld32(tmem_row + tmem_dK + c * 32, rk);
-        tmem_ld32(tmem_row + tmem_dV + c * 32, rv);
-        tmem_ld_wait();
-      } else {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) { rk[e] = 0; rv[e] = 0; }
-      }
-      if (r_ok) {
-        float v[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rk[e]) * p.scale;
-        store_row_chunk32(dks, c * 32, 1, v);
-#pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rv[e]);
-        store_row_chunk32(dvs, c * 32, 1, v);
+    } else if (warp >= 2) {
+      // ---------------- row statistics ----------------
+      const int i = tid - 64;  // 0..63
+      for (int it = 0; it < n_it; ++it) {
+        const int st = it % NSTQ;
+        const int q = q0_of(it) + i;
+        const float2 v = (q < p.L) ? p.stats[size_t(q_plane_of(it)) * p.L + q]
+                                   : make_float2(INFINITY, 0.f);
+        if (it >= NSTQ) wait(bar_qe + st, (it / NSTQ - 1) & 1);
+        s_stat[st * 64 + i] = make_float2(-v.x, v.y);
+        mbar_arrive(bar_sf + st);
       }
     }
   } else {
-    // final rows: window part plus, for initial/separator tokens, the side partial of the same token
-    const bool r_ok = key < p.L;
-    int side_idx = -1;
-    if (r_ok) {
-      const int32_t* cnt_b = p.cnt + size_t(b) * (p.L + 1);
-      const int c0 = cnt_b[key], c1 = cnt_b[key + 1];
-      if (c1 > c0 && c0 < ns) {
-        // the side pass wrote this row only if some query sees it from outside its window
-        const int t_first = (key + p.n_neighbor) / kBM;
-        if (t_first <= p.T - 1) side_idx = c0;
-      }
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    // ---------------- P^T and dS^T ----------------
+    const int u = (warp >= 8) ? 1 : 0;
+    const int r = tid & 127;
+    const int key = kt * kBN + r;  // side entry index (SIDE) or key position (window)
+    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+    const uint32_t tb = tmem + lane_base + C::kBuf + u * C::kBufStride;
+    // queries that keep this key: [q_first, q_first + span)
+    int q_first, span, tile_q_max;
+    if (SIDE) {
+      q_first = (key < ns) ? p.side_pos[size_t(b) * p.side_cap + key] + p.n_neighbor : kFar;
+      span = kFar;
+      // first query that keeps every key of the tile (never, if the tile has padding rows)
+      tile_q_max = (kt * kBN + kBN <= ns)
+                       ? p.side_pos[size_t(b) * p.side_cap + kt * kBN + kBN - 1] + p.n_neighbor
+                       : kFar;
+    } else {
+      q_first = key;
+      span = p.n_neighbor;
+      tile_q_max = 0;
     }
-    const float* dks = p.dKs + (size_t(kv_plane) * p.cap_pad + max(side_idx, 0)) * D;
-    const float* dvs = p.dVs + (size_t(kv_plane) * p.cap_pad + max(side_idx, 0)) * D;
+    for (int it = u; it < n_it; it += 2) {
+      const int st = it % NSTQ;
+      const int q0 = q0_of(it);
+      const int c_lo = q_first - q0, c_hi = c_lo + span;
+      bool need_mask;
+      if (SIDE) need_mask = tile_q_max > q0;
+      else need_mask = !(kt * kBN + kBN - 1 <= q0 && q0 + 63 <= kt * kBN + p.n_neighbor - 1);
+      wait(bar_sf + st, (it / NSTQ) & 1);
+      wait(bar_sp + u, (it >> 1) & 1);
+      tc_fence_after();
+      const float2* stat = s_stat + st * 64;
+      uint32_t pkp[32], pkd[32];
 #pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t rk[32], rv[32];
-      tmem_ld32(tmem_row + tmem_dK + c * 32, rk);
-      tmem_ld32(tmem_row + tmem_dV + c * 32, rv);
-      tmem_ld_wait();
+      for (int c = 0; c < 2; ++c) {
+        uint32_t sv[32], dp[32];
+        tmem_ld32(tb + C::kST + c * 32, sv);
+        tmem_ld32(tb + C::kdPT + c * 32, dp);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          float pr[2], ds[2];
+#pragma unroll
+          for (int w = 0; w < 2; ++w) {
+            const int col = c * 32 + e + w;
+            const float2 sd = stat[col];  // (-LSE in log2 units, Delta)
+            pr[w] = ex2(fmaf(__uint_as_float(sv[e + w]), p.scale_log2, sd.x));
+            if (need_mask && !(col >= c_lo && col < c_hi)) pr[w] = 0.f;
+            ds[w] = pr[w] * (__uint_as_float(dp[e + w]) - sd.y);
+          }
+          pkp[c * 16 + (e >> 1)] = pack_bf16(pr[0], pr[1]);
+          pkd[c * 16 + (e >> 1)] = pack_bf16(ds[0], ds[1]);
+        }
+      }
+      tmem_st32(tb + C::kST, pkp);
+      tmem_st32(tb + C::kdPT, pkd);
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar_pds + u);
+    }
+
+    // ---------------- epilogue: warps 4-7 take dV, warps 8-11 take dK ----------------
+    if (n_it > 0) {
+      wait(bar_acc, 0);
+      tc_fence_after();
+    }
+    const uint32_t t_acc = tmem + lane_base + (u ? C::kdK : C::kdV);
+    const float mul = u ? p.scale : 1.f;
+    if (SIDE) {
+      // fp32 partial rows for the entries of this side tile
+      const bool r_ok = key < p.cap_pad;
+      float* base = (u ? p.dKs : p.dVs) +
+                    ((size_t(part) * gridDim.z + b) * p.Hkv + hk) * size_t(p.cap_pad) * D +
+                    size_t(key) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t rr[32];
+        if (n_it > 0) {
+          tmem_ld32(t_acc + c * 32, rr);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) rr[e] = 0;
+        }
+        if (r_ok) {
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * mul;
+          store_row_chunk32(base, c * 32, 1, v);
+        }
+      }
+    } else {
+      // final rows: window part plus, for initial/separator tokens, the side partials of the token
+      const bool r_ok = key < p.L;
+      int side_idx = -1;
       if (r_ok) {
-        float v[32];
+        const int32_t* cnt_b = p.cnt + size_t(b) * (p.L + 1);
+        const int c0 = cnt_b[key], c1 = cnt_b[key + 1];
+        if (c1 > c0 && c0 < ns) side_idx = c0;
+      }
+      const size_t part_stride = size_t(gridDim.z) * p.Hkv * size_t(p.cap_pad) * D;
+      const float* part0 = (u ? p.dKs : p.dVs) +
+                           (size_t(b) * p.Hkv + hk) * size_t(p.cap_pad) * D +
+                           size_t(max(side_idx, 0)) * D;
+      void* out = u ? p.dK : p.dV;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rk[e]) * p.scale;
-        if (side_idx >= 0) {
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t rr[32];
+        tmem_ld32(t_acc + c * 32, rr);
+        tmem_ld_wait();
+        if (r_ok) {
+          float v[32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] += dks[c * 32 + e];
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * mul;
+          if (side_idx >= 0) {
+            for (int sp = 0; sp < p.split; ++sp) {
+              const float4* src = reinterpret_cast<const float4*>(part0 + sp * part_stride + c * 32);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 a = src[q];
+                v[4 * q] += a.x; v[4 * q + 1] += a.y; v[4 * q + 2] += a.z; v[4 * q + 3] += a.w;
+              }
+            }
+          }
+          store_row_chunk32(out, (size_t(kv_plane) * p.L + key) * D + c * 32, p.grad_fp32, v);
         }
-        store_row_chunk32(p.dK, (size_t(kv_plane) * p.L + key) * D + c * 32, p.grad_fp32, v);
-#pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rv[e]);
-        if (side_idx >= 0) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] += dvs[c * 32 + e];
-        }
-        store_row_chunk32(p.dV, (size_t(kv_plane) * p.L + key) * D + c * 32, p.grad_fp32, v);
       }
     }
   }
@@ -626,26 +702,33 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
     launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
   record_event(d, 1, stream);
 
-  float* delta = reinterpret_cast<float*>(ws + lay.off_delta);
+  float2* stats = reinterpret_cast<float2*>(ws + lay.off_delta);
   const size_t rows = size_t(d->B) * d->Hq * d->L;
   {
     constexpr int RPB = 256 / (D / 8);
     bwd_delta<D><<<unsigned((rows + RPB - 1) / RPB), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(dO), static_cast<const __nv_bfloat16*>(O), delta, rows);
+        static_cast<const __nv_bfloat16*>(dO), static_cast<const __nv_bfloat16*>(O), LSE, stats,
+        rows);
   }
   record_event(d, 2, stream);
 
-  CUtensorMap mq, mdo, mk, mv, mks, mvs;
+  // 128-row boxes for the stationary operand of each pass, 64-row boxes for the streamed one
+  CUtensorMap mq, mdo, mk, mv, mks, mvs, mq_h, mdo_h, mk_h, mv_h, mks_h, mvs_h;
   sepllm_status st;
-  const int64_t L = d->L;
-  if ((st = make_tile_map(&mq, Q, D, L, int64_t(d->B) * d->Hq, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mdo, dO, D, L, int64_t(d->B) * d->Hq, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mk, K, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mv, V, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mks, Ks, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
-                          int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mvs, Vs, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
-                          int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
+  const int64_t L = d->L, nq = int64_t(d->B) * d->Hq, nkv = int64_t(d->B) * d->Hkv;
+  const int64_t cp = lay.cap_pad;
+  if ((st = make_tile_map(&mq, Q, D, L, nq, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mdo, dO, D, L, nq, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mk, K, D, L, nkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mv, V, D, L, nkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mks, Ks, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mvs, Vs, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mq_h, Q, D, L, nq, D, L * D, 64)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mdo_h, dO, D, L, nq, D, L * D, 64)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mk_h, K, D, L, nkv, D, L * D, 64)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mv_h, V, D, L, nkv, D, L * D, 64)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mks_h, Ks, D, cp, nkv, D, cp * D, 64)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mvs_h, Vs, D, cp, nkv, D, cp * D, 64)) != SEPLLM_OK) return st;
 
   BwdParams p;
   p.cnt = reinterpret_cast<const int32_t*>(index + ih.off_cnt);
@@ -653,8 +736,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.side_pos = side_pos;
   p.n_side = n_side;
   p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
-  p.LSE = LSE;
-  p.delta = delta;
+  p.stats = stats;
   p.dKs = reinterpret_cast<float*>(ws + lay.off_dks);
   p.dVs = reinterpret_cast<float*>(ws + lay.off_dvs);
   p.dQ = dQ;
@@ -669,25 +751,30 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.side_cap = id->side_cap;
   p.cap_pad = lay.cap_pad;
   p.grad_fp32 = d->grad_dtype;
+  p.split = lay.split;
+  const int G = d->Hq / d->Hkv;
+  p.pair_heads = (G % 2 == 0) ? 1 : 0;
   p.scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
   p.scale_log2 = p.scale * kLog2e;
 
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       int(DqSmem<D>::kRequest)));
+                                       int(DqCfg<D>::kRequest)));
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, true>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       int(DkvSmem<D>::kRequest)));
+                                       int(DkvCfg<D>::kRequest)));
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       int(DkvSmem<D>::kRequest)));
-  bwd_dq_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), 128, DqSmem<D>::kRequest, stream>>>(
-      mq, mdo, mk, mv, mks, mvs, p);
+                                       int(DkvCfg<D>::kRequest)));
+  const dim3 grid_dq = p.pair_heads ? dim3(ih.n_tiles, d->Hq / 2, d->B)
+                                    : dim3((ih.n_tiles + 1) / 2, d->Hq, d->B);
+  bwd_dq_kernel<D><<<grid_dq, kBwdThreads, DqCfg<D>::kRequest, stream>>>(mq, mdo, mk_h, mv_h, mks_h,
+                                                                         mvs_h, p);
   record_event(d, 3, stream);
-  bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv, d->B), 128, DkvSmem<D>::kRequest,
-                            stream>>>(mq, mdo, mks, mvs, p);
+  bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv * lay.split, d->B), kBwdThreads,
+                            DkvCfg<D>::kRequest, stream>>>(mq_h, mdo_h, mks, mvs, p);
   record_event(d, 4, stream);
-  bwd_dkv_kernel<D, false><<<dim3(ih.n_tiles, d->Hkv, d->B), 128, DkvSmem<D>::kRequest, stream>>>(
-      mq, mdo, mk, mv, p);
+  bwd_dkv_kernel<D, false><<<dim3(ih.n_tiles, d->Hkv, d->B), kBwdThreads, DkvCfg<D>::kRequest,
+                             stream>>>(mq_h, mdo_h, mk, mv, p);
   record_event(d, 5, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;

@@ -11,8 +11,10 @@ struct AttnLayout {
   int cap_pad;  // side_cap rounded up to 128 rows
   // forward workspace: status | Kside | Vside
   size_t off_ks, off_vs, fwd_bytes;
-  // backward workspace: status | Kside | Vside | Delta | dKside | dVside
+  // backward workspace: status | Kside | Vside | row statistics (LSE in log2 units, Delta) |
+  // dKside | dVside, the last two fp32 [split][B][Hkv][cap_pad][d]
   size_t off_delta, off_dks, off_dvs, bwd_bytes;
+  int split;
 };
 
 sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id);

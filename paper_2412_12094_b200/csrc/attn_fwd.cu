@@ -118,19 +118,6 @@ struct FwdParams {
   float scale_log2;
 };
 
-// D[tmem] (+)= A[tmem, packed bf16] * B[smem]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc,
-                                        uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
@@ -455,8 +442,10 @@ AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
   a.off_vs = a.off_ks + side_bytes;
   a.fwd_bytes = a.off_vs + side_bytes;
   a.off_delta = a.fwd_bytes;
-  a.off_dks = a.off_delta + align_up(size_t(d->B) * d->Hq * d->L * sizeof(float));
-  const size_t side_grad = align_up(size_t(d->B) * d->Hkv * a.cap_pad * d->d * sizeof(float));
+  a.off_dks = a.off_delta + align_up(size_t(d->B) * d->Hq * d->L * 2 * sizeof(float));
+  a.split = d->Hq / d->Hkv;  // one side-gradient partial per query head of a group
+  const size_t side_grad =
+      align_up(size_t(a.split) * d->B * d->Hkv * a.cap_pad * d->d * sizeof(float));
   a.off_dvs = a.off_dks + side_grad;
   a.bwd_bytes = a.off_dvs + side_grad;
   return a;

@@ -138,41 +138,21 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
-  int t_x[2], hq_x[2];
+  SlotGeom g0, g1;
   if (p.pair_heads) {
-    t_x[0] = t_x[1] = p.T - 1 - int(blockIdx.x);
-    hq_x[0] = 2 * int(blockIdx.y);
-    hq_x[1] = hq_x[0] + 1;
+    const int t = p.T - 1 - int(blockIdx.x);
+    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y), p.cap_pad / kBN);
+    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y) + 1, p.cap_pad / kBN);
   } else {
-    t_x[1] = p.T - 1 - 2 * int(blockIdx.x);
-    t_x[0] = t_x[1] - 1;
-    hq_x[0] = hq_x[1] = int(blockIdx.y);
+    const int t = p.T - 1 - 2 * int(blockIdx.x);
+    g0 = load_slot(p.tile_meta, b, p.T, t - 1, int(blockIdx.y), p.cap_pad / kBN);
+    g1 = load_slot(p.tile_meta, b, p.T, t, int(blockIdx.y), p.cap_pad / kBN);
   }
-  const int kv_plane = b * p.Hkv + hq_x[0] / G;
-  int side_full_x[2], ns_x[2], wlo_x[2], whi_x[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    if (t_x[x] >= 0) {
-      const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t_x[x]) * 8;
-      side_full_x[x] = meta[0];
-      ns_x[x] = min(meta[1], p.cap_pad / kBN);
-      wlo_x[x] = meta[4];
-      whi_x[x] = meta[5];
-    } else {
-      side_full_x[x] = 0; ns_x[x] = 0; wlo_x[x] = 0; whi_x[x] = 0;
-    }
-  }
-  if (t_x[0] < 0) { wlo_x[0] = wlo_x[1]; whi_x[0] = wlo_x[1]; }
-  const int ns = max(ns_x[0], ns_x[1]);
-  const int wlo = min(wlo_x[0], wlo_x[1]);
-  const int whi = max(whi_x[0], whi_x[1]);
+  const int kv_plane = b * p.Hkv + g1.hq / G;
+  const int ns = max(g0.ns, g1.ns);
+  const int wlo = min(g0.wlo, g1.wlo);
+  const int whi = max(g0.whi, g1.whi);
   const int n_steps = 2 * (ns + (whi - wlo));  // key half-tiles
-  auto active = [&](int x, int s) -> bool {
-    const int j = s >> 1;
-    if (j < ns) return j < ns_x[x];
-    const int w = wlo + (j - ns);
-    return w >= wlo_x[x] && w < whi_x[x];
-  };
   // first key row of half-tile s in its tensor (side buffer or K/V)
   auto half_y = [&](int s) -> int {
     const int j = s >> 1;
@@ -206,20 +186,22 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   };
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
 #pragma unroll
-      for (int x = 0; x < 2; ++x)
-        if (t_x[x] >= 0) {
+      for (int x = 0; x < 2; ++x) {
+        const SlotGeom& g = x ? g1 : g0;
+        if (g.t >= 0) {
           mbar_expect_tx(bar_q + x, 2 * C::kTile);
           for (int nb = 0; nb < NB; ++nb) {
             tma_load_3d(sQ + x * C::kTile + nb * kTileBlockBytes, &mapQ, bar_q + x, nb * 64,
-                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+                        g.t * kBM, b * p.Hq + g.hq);
             tma_load_3d(sdO + x * C::kTile + nb * kTileBlockBytes, &mapdO, bar_q + x, nb * 64,
-                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+                        g.t * kBM, b * p.Hq + g.hq);
           }
         }
+      }
       for (int s = 0; s < n_steps; ++s) {
         const bool side = (s >> 1) < ns;
         const int y = half_y(s);
@@ -239,45 +221,45 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t q_lo[2] = {desc_lo(smem_u32(sQ), 16), desc_lo(smem_u32(sQ + C::kTile), 16)};
+      const uint32_t do_lo[2] = {desc_lo(smem_u32(sdO), 16), desc_lo(smem_u32(sdO + C::kTile), 16)};
+      const uint32_t k_lo0 = desc_lo(smem_u32(sK), 16);                  // K_h as the K-major B of S
+      const uint32_t kt_lo0 = desc_lo(smem_u32(sK), kHalfBlockBytes);    // K_h as the MN-major B of dQ
+      const uint32_t v_lo0 = desc_lo(smem_u32(sV), 16);
       int n_dq[2] = {0, 0};
       bool q_seen[2] = {false, false};
       for (int s = 0; s <= n_steps; ++s) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
+          const SlotGeom& g = x ? g1 : g0;
           const uint32_t tb = tmem + x * C::kSlot;
-          if (s >= 1 && active(x, s - 1)) {
+          if (s >= 1 && slot_active(g, ns, wlo, (s - 1) >> 1)) {
             const int sk = (s - 1) % NSK;
             wait(bar_ds + x, n_dq[x] & 1);
             tc_fence_after();
-            const uint32_t ka = smem_u32(sK + sk * C::kHalf);
+            const uint32_t kt_lo = kt_lo0 + sk * (C::kHalf >> 4);
+            umma_ts_lo(tb + C::kdQ, tb + C::kS, kt_lo, idesc_dq, n_dq[x] > 0);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_ts(tb + C::kdQ, tb + C::kS + k * 8,
-                      make_smem_desc(ka + k * 2048, kHalfBlockBytes, 1024), idesc_dq,
-                      (n_dq[x] > 0 || k > 0));
+            for (int k = 1; k < 4; ++k)
+              umma_ts_lo(tb + C::kdQ, tb + C::kS + k * 8, kt_lo + mnmajor_step(k), idesc_dq, 1);
             ++n_dq[x];
           }
-          if (s < n_steps && active(x, s)) {
+          if (s < n_steps && slot_active(g, ns, wlo, s >> 1)) {
             const int sk = s % NSK, sv = s % NSV;
             if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
             wait(bar_kf + sk, (s / NSK) & 1);
             tc_fence_after();
-            const uint32_t qa = smem_u32(sQ + x * C::kTile), doa = smem_u32(sdO + x * C::kTile);
-            const uint32_t ka = smem_u32(sK + sk * C::kHalf), va = smem_u32(sV + sv * C::kHalf);
+            const uint32_t k_lo = k_lo0 + sk * (C::kHalf >> 4), v_lo = v_lo0 + sv * (C::kHalf >> 4);
 #pragma unroll
             for (int k = 0; k < D / 16; ++k)
-              umma_ss(tb + C::kS,
-                      make_smem_desc(qa + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
-                      make_smem_desc(ka + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024),
-                      idesc_s, k > 0);
+              umma_ss_lo(tb + C::kS, q_lo[x] + kmajor_step(k, kTileBlockBytes),
+                         k_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
             wait(bar_vf + sv, (s / NSV) & 1);
             tc_fence_after();
 #pragma unroll
             for (int k = 0; k < D / 16; ++k)
-              umma_ss(tb + C::kdP,
-                      make_smem_desc(doa + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
-                      make_smem_desc(va + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024),
-                      idesc_s, k > 0);
+              umma_ss_lo(tb + C::kdP, do_lo[x] + kmajor_step(k, kTileBlockBytes),
+                         v_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
             tc_commit(bar_sp + x);
           }
         }
@@ -287,23 +269,24 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       tc_commit(bar_acc);
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ---------------- dS of slot x ----------------
     const int x = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;
     const uint32_t tb = tmem + (uint32_t((warp & 3) * 32) << 16) + x * C::kSlot;
-    const int t = t_x[x];
+    const SlotGeom g = x ? g1 : g0;
+    const int t = g.t;
     if (t >= 0) {
       const int row = t * kBM + r;
       const bool row_ok = row < p.L;
-      const int q_plane = b * p.Hq + hq_x[x];
+      const int q_plane = b * p.Hq + g.hq;
       const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
       const float2 st = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
       const float neg_lse2 = -st.x, delta_i = st.y;
-      const int side_full = side_full_x[x];
+      const int side_full = g.side_full;
       int n_done = 0;
       for (int s = 0; s < n_steps; ++s) {
-        if (!active(x, s)) continue;
+        if (!slot_active(g, ns, wlo, s >> 1)) continue;
         const int j = s >> 1;
         const bool side = j < ns;
         int c_lo = 0, c_hi = 64;
@@ -473,7 +456,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   auto q0_of = [&](int it) { return (qh_lo + it / n_g) * 64; };
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 0 && lane == 0 && n_it > 0) {
       // ---------------- TMA producer ----------------
       mbar_expect_tx(bar_kv, 2 * C::kTile);
@@ -496,25 +479,23 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
       constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t ka = smem_u32(sK), va = smem_u32(sV);
+      const uint32_t k_lo = desc_lo(smem_u32(sK), 16), v_lo = desc_lo(smem_u32(sV), 16);
+      const uint32_t q_lo0 = desc_lo(smem_u32(sQ), 16);                   // Q_h, dO_h as K-major B
+      const uint32_t qt_lo0 = desc_lo(smem_u32(sQ), kHalfBlockBytes);     // ... as MN-major B
       auto issue_sp = [&](int it) {
         const int st = it % NSTQ, u = it & 1;
         wait(bar_qf + st, (it / NSTQ) & 1);
         tc_fence_after();
-        const uint32_t qa = smem_u32(sQ + st * 2 * C::kHalf), doa = qa + C::kHalf;
+        const uint32_t q_lo = q_lo0 + st * (2 * C::kHalf >> 4), do_lo = q_lo + (C::kHalf >> 4);
         const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          umma_ss(tb + C::kST,
-                  make_smem_desc(ka + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
-                  make_smem_desc(qa + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024), idesc_s,
-                  k > 0);
+          umma_ss_lo(tb + C::kST, k_lo + kmajor_step(k, kTileBlockBytes),
+                     q_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          umma_ss(tb + C::kdPT,
-                  make_smem_desc(va + (k / 4) * kTileBlockBytes + (k % 4) * 32, 16, 1024),
-                  make_smem_desc(doa + (k / 4) * kHalfBlockBytes + (k % 4) * 32, 16, 1024), idesc_s,
-                  k > 0);
+          umma_ss_lo(tb + C::kdPT, v_lo + kmajor_step(k, kTileBlockBytes),
+                     do_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
         tc_commit(bar_sp + u);
       };
       wait(bar_kv, 0);
@@ -524,16 +505,16 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int st = it % NSTQ, u = it & 1;
         wait(bar_pds + u, (it >> 1) & 1);
         tc_fence_after();
-        const uint32_t qa = smem_u32(sQ + st * 2 * C::kHalf), doa = qa + C::kHalf;
+        const uint32_t qt_lo = qt_lo0 + st * (2 * C::kHalf >> 4), dot_lo = qt_lo + (C::kHalf >> 4);
         const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
+        umma_ts_lo(tmem + C::kdV, tb + C::kST, dot_lo, idesc_acc, it > 0);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + C::kdV, tb + C::kST + k * 8,
-                  make_smem_desc(doa + k * 2048, kHalfBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
+        for (int k = 1; k < 4; ++k)
+          umma_ts_lo(tmem + C::kdV, tb + C::kST + k * 8, dot_lo + mnmajor_step(k), idesc_acc, 1);
+        umma_ts_lo(tmem + C::kdK, tb + C::kdPT, qt_lo, idesc_acc, it > 0);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + C::kdK, tb + C::kdPT + k * 8,
-                  make_smem_desc(qa + k * 2048, kHalfBlockBytes, 1024), idesc_acc, (it > 0 || k > 0));
+        for (int k = 1; k < 4; ++k)
+          umma_ts_lo(tmem + C::kdK, tb + C::kdPT + k * 8, qt_lo + mnmajor_step(k), idesc_acc, 1);
         tc_commit(bar_qe + st);
         if (it + 2 < n_it) issue_sp(it + 2);
       }
@@ -552,7 +533,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ---------------- P^T and dS^T ----------------
     const int u = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;

@@ -7,6 +7,34 @@ namespace sepllm {
 constexpr int kBM = 128, kBN = 128;
 constexpr uint32_t kTileBlockBytes = 128 * 128;  // 128 rows x 64 bf16, one swizzled block
 
+// One query tile of a two-slot CTA (forward and dQ kernels): tile index (-1 = empty slot), query
+// head, and the tile's key ranges from tile_meta.
+struct SlotGeom {
+  int t, hq, side_full, ns, wlo, whi;
+};
+__device__ __forceinline__ SlotGeom load_slot(const int32_t* tile_meta, int b, int T, int t, int hq,
+                                              int side_tiles_cap) {
+  SlotGeom g;
+  g.t = t;
+  g.hq = hq;
+  if (t >= 0) {
+    const int32_t* meta = tile_meta + (size_t(b) * T + t) * 8;
+    g.side_full = meta[0];
+    g.ns = min(meta[1], side_tiles_cap);
+    g.wlo = meta[4];
+    g.whi = meta[5];
+  } else {
+    g.side_full = 0; g.ns = 0; g.wlo = 0x3fffffff; g.whi = 0;
+  }
+  return g;
+}
+// Key tile j of the CTA's list (side tiles [0, ns), then window tiles from wlo) is kept by slot g.
+__device__ __forceinline__ bool slot_active(const SlotGeom& g, int ns, int wlo, int j) {
+  if (j < ns) return j < g.ns;
+  const int w = wlo + (j - ns);
+  return w >= g.wlo && w < g.whi;
+}
+
 struct AttnLayout {
   int cap_pad;  // side_cap rounded up to 128 rows
   // forward workspace: status | Kside | Vside

@@ -148,41 +148,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   const int G = p.Hq / p.Hkv;
 
   // the two slots of this CTA (slot 1 is never empty; slot 0 is when T is odd and tiles pair up)
-  int t_x[2], hq_x[2];
+  SlotGeom g0, g1;
   if (p.pair_heads) {
-    t_x[0] = t_x[1] = p.T - 1 - int(blockIdx.x);  // long tiles first
-    hq_x[0] = 2 * int(blockIdx.y);
-    hq_x[1] = hq_x[0] + 1;
+    const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
+    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y), p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y) + 1, p.side_tiles_cap);
   } else {
-    t_x[1] = p.T - 1 - 2 * int(blockIdx.x);
-    t_x[0] = t_x[1] - 1;
-    hq_x[0] = hq_x[1] = int(blockIdx.y);
+    const int t = p.T - 1 - 2 * int(blockIdx.x);
+    g0 = load_slot(p.tile_meta, b, p.T, t - 1, int(blockIdx.y), p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, b, p.T, t, int(blockIdx.y), p.side_tiles_cap);
   }
-  const int kv_plane = b * p.Hkv + hq_x[0] / G;
-  int side_full_x[2], ns_x[2], wlo_x[2], whi_x[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    if (t_x[x] >= 0) {
-      const int32_t* meta = p.tile_meta + (size_t(b) * p.T + t_x[x]) * 8;
-      side_full_x[x] = meta[0];
-      ns_x[x] = min(meta[1], p.side_tiles_cap);
-      wlo_x[x] = meta[4];
-      whi_x[x] = meta[5];
-    } else {
-      side_full_x[x] = 0; ns_x[x] = 0; wlo_x[x] = wlo_x[1 - x]; whi_x[x] = wlo_x[x];
-    }
-  }
-  if (t_x[0] < 0) { wlo_x[0] = wlo_x[1]; whi_x[0] = wlo_x[1]; }
+  const int kv_plane = b * p.Hkv + g1.hq / G;
   // key tiles of the CTA: side tiles [0, ns), then window tiles [wlo, whi)
-  const int ns = max(ns_x[0], ns_x[1]);
-  const int wlo = min(wlo_x[0], wlo_x[1]);
-  const int whi = max(whi_x[0], whi_x[1]);
+  const int ns = max(g0.ns, g1.ns);
+  const int wlo = min(g0.wlo, g1.wlo);
+  const int whi = max(g0.whi, g1.whi);
   const int n_tiles = ns + (whi - wlo);
-  auto active = [&](int x, int j) -> bool {
-    if (j < ns) return j < ns_x[x];
-    const int w = wlo + (j - ns);
-    return w >= wlo_x[x] && w < whi_x[x];
-  };
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_s + i, 1); mbar_init(bar_p + i, 128); }
@@ -214,17 +195,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   };
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
 #pragma unroll
-      for (int x = 0; x < 2; ++x)
-        if (t_x[x] >= 0) {
+      for (int x = 0; x < 2; ++x) {
+        const SlotGeom& g = x ? g1 : g0;
+        if (g.t >= 0) {
           mbar_expect_tx(bar_q + x, C::kTile);
           for (int nb = 0; nb < NB; ++nb)
             tma_load_3d(sQ + x * C::kTile + nb * kTileBlockBytes, &mapQ, bar_q + x, nb * 64,
-                        t_x[x] * kBM, b * p.Hq + hq_x[x]);
+                        g.t * kBM, b * p.Hq + g.hq);
         }
+      }
       for (int j = 0; j < n_tiles; ++j) {
         const int st = j % NST, use = j / NST;
         const bool side = j < ns;
@@ -244,36 +227,38 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t q_lo[2] = {desc_lo(smem_u32(sQ), 16), desc_lo(smem_u32(sQ + C::kTile), 16)};
+      const uint32_t k_lo0 = desc_lo(smem_u32(sK), 16);
+      const uint32_t v_lo0 = desc_lo(smem_u32(sV), kTileBlockBytes);
       int n_pv[2] = {0, 0};  // PV MMAs issued per slot
       bool q_seen[2] = {false, false};
       for (int s = 0; s <= n_tiles; ++s) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
+          const SlotGeom& g = x ? g1 : g0;
           const uint32_t tS = tmem + (x ? C::kS1 : C::kS0), tO = tmem + (x ? C::kO1 : C::kO0);
-          if (s >= 1 && active(x, s - 1)) {
+          if (s >= 1 && slot_active(g, ns, wlo, s - 1)) {
             const int j = s - 1, st = j % NST;
             wait(bar_p + x, n_pv[x] & 1);
             wait(bar_vf + st, (j / NST) & 1);
             tc_fence_after();
-            const uint32_t va = smem_u32(sV + st * C::kTile);
+            const uint32_t v_lo = v_lo0 + st * (C::kTile >> 4);
+            umma_ts_lo(tO, tS, v_lo, idesc_o, n_pv[x] > 0);
 #pragma unroll
-            for (int k = 0; k < kBN / 16; ++k)
-              umma_ts(tO, tS + k * 8, make_smem_desc(va + k * 2048, kTileBlockBytes, 1024), idesc_o,
-                      (n_pv[x] > 0 || k > 0));
+            for (int k = 1; k < kBN / 16; ++k)
+              umma_ts_lo(tO, tS + k * 8, v_lo + mnmajor_step(k), idesc_o, 1);
             ++n_pv[x];
           }
-          if (s < n_tiles && active(x, s)) {
+          if (s < n_tiles && slot_active(g, ns, wlo, s)) {
             const int st = s % NST;
             if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
             wait(bar_kf + st, (s / NST) & 1);
             tc_fence_after();
-            const uint32_t qa = smem_u32(sQ + x * C::kTile), ka = smem_u32(sK + st * C::kTile);
+            const uint32_t k_lo = k_lo0 + st * (C::kTile >> 4);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-              const uint32_t off = (k / 4) * kTileBlockBytes + (k % 4) * 32;
-              umma_ss(tS, make_smem_desc(qa + off, 16, 1024), make_smem_desc(ka + off, 16, 1024),
-                      idesc_s, k > 0);
-            }
+            for (int k = 0; k < D / 16; ++k)
+              umma_ss_lo(tS, q_lo[x] + kmajor_step(k, kTileBlockBytes),
+                         k_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
             tc_commit(bar_s + x);
           }
         }
@@ -283,25 +268,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       tc_commit(bar_o);
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ---------------- softmax of slot x ----------------
     const int x = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;                       // row in the tile = tensor-memory lane
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + (x ? C::kS1 : C::kS0);
     const uint32_t tO = tmem + lane_base + (x ? C::kO1 : C::kO0);
-    const int t = t_x[x];
+    const SlotGeom g = x ? g1 : g0;
+    const int t = g.t;
     if (t >= 0) {
       const int row = t * kBM + r;  // this thread's query position
-      const int q_plane = b * p.Hq + hq_x[x];
+      const int q_plane = b * p.Hq + g.hq;
       const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-      const int side_full = side_full_x[x];
+      const int side_full = g.side_full;
       float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
       float l_sum = 0.f;
       int n_done = 0;
       uint32_t sreg[4][32];
       for (int j = 0; j < n_tiles; ++j) {
-        if (!active(x, j)) continue;
+        if (!slot_active(g, ns, wlo, j)) continue;
         wait(bar_s + x, n_done & 1);
         tc_fence_after();
 #pragma unroll

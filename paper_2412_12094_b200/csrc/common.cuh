@@ -150,19 +150,6 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_
       : "memory");
 }
 
-// D[tmem] (+)= A[tmem, packed bf16] * B[smem]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc,
-                                        uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 // Shared-memory matrix descriptor, 128-byte swizzle, tile base 1024-byte aligned.
 //   K-major operand  (rows of 64 bf16 along the contraction): SBO = 1024 (8 rows), LBO unused.
 //   MN-major operand (rows of 64 bf16 along M or N, one row per contraction index):
@@ -177,6 +164,50 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
   d |= static_cast<uint64_t>(2) << 61;  // 128-byte swizzle
   return d;
 }
+
+// The MMA-issuing thread is a single thread with a long dependent instruction stream, so its
+// descriptors are built from a per-tile low word plus compile-time offsets: every descriptor used
+// here has the same high word (SBO 1024, version 1, 128-byte swizzle) and a low word of
+// (address >> 4) | (LBO >> 4) << 16; offsets inside a tile never carry out of the address field.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+// D[tmem] (+)= A[smem] * B[smem] from descriptor low words
+__device__ __forceinline__ void umma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                           uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      ".reg .b64 da, db;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "mov.b64 da, {%1, %5};\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem, packed bf16: column c holds contraction indices 2c, 2c+1] * B[smem]
+__device__ __forceinline__ void umma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
+                                           uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      ".reg .b64 db;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+      : "memory");
+}
+// 16-byte units to step a K-major operand (rows of 64 bf16, blocks of `block_bytes`) by 16
+// contraction indices k times, and an MN-major operand by 16 contraction rows k times
+__device__ __forceinline__ constexpr uint32_t kmajor_step(int k, uint32_t block_bytes) {
+  return uint32_t(k / 4) * (block_bytes >> 4) + uint32_t(k % 4) * 2u;
+}
+__device__ __forceinline__ constexpr uint32_t mnmajor_step(int k) { return uint32_t(k) * 128u; }
 
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 D.
 // a_mn / b_mn: 1 when that operand is MN-major in shared memory.

@@ -86,73 +86,61 @@ constexpr int kFar = 0x3fffffff;                // "never" / "unbounded" for col
 // ---------------------------------------------------------------------------
 // dQ: query-tile stationary
 // ---------------------------------------------------------------------------
-// Same shape as the forward: two query-tile slots per CTA sharing their key tiles, a TMA warp, an
-// MMA warp and one arithmetic warpgroup per slot.  Keys are taken 64 at a time so that a slot's
-// S, dP (64 columns each) and dQ (D columns) fit in half of tensor memory:
-//   S_x = Q_x K_h^T, dP_x = dO_x V_h^T  ->  dS = P (dP - Delta) written as packed bf16 over S_x
-//   dQ_x += dS K_h  (A operand from tensor memory).
+// One CTA owns one query tile of one head.  Shared-memory bandwidth is what bounds these MMAs, so
+// the stationary operands Q and dO are kept in tensor memory (packed bf16, written once by the
+// arithmetic threads straight from global memory) and only the streamed K_h / V_h half-tiles of
+// 64 keys pass through shared memory:
+//   warp 0      TMA producer: [K_h | V_h] stages of a ring
+//   warp 1      MMA issuer:   S = Q K_h^T and dP = dO V_h^T into one of two buffers (A from tensor
+//               memory), later dQ += dS K_h with dS read from the buffer it was computed in
+//   warps 4-7   dS = P (dP - Delta) of even half-tiles (thread = query row), packed bf16 over S
+//   warps 8-11  the same for odd half-tiles
 template <int D>
 struct DqCfg {
   static constexpr int NB = D / 64;
-  static constexpr int NSK = 3, NSV = 2;            // K_h is read by two consecutive steps
-  static constexpr uint32_t kTile = NB * kTileBlockBytes;
-  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;
-  static constexpr uint32_t kQ = 0;                 // Q_0, Q_1
-  static constexpr uint32_t kdO = kQ + 2 * kTile;   // dO_0, dO_1
-  static constexpr uint32_t kK = kdO + 2 * kTile;
-  static constexpr uint32_t kV = kK + NSK * kHalf;
-  static constexpr uint32_t kBar = kV + NSV * kHalf;
+  static constexpr int NST = 5;
+  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;   // one 64-key half-tile of K or V
+  static constexpr uint32_t kStage = 2 * kHalf;
+  static constexpr uint32_t kKV = 0;
+  static constexpr uint32_t kBar = kKV + NST * kStage;
   static constexpr uint32_t kTotal = kBar + 512;
   static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
-  // tensor-memory columns: per slot S (64) | dP (64) | dQ (D)
-  static constexpr uint32_t kSlot = 256, kS = 0, kdP = 64, kdQ = 128;
+  // tensor-memory columns
+  static constexpr uint32_t kQt = 0, kdOt = 64, kBuf = 128, kBufStride = 128, kS = 0, kdP = 64,
+                            kdQ = 384;
 };
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
-bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
-              const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
               const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
+              const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ dOg,
               const BwdParams p) {
   using C = DqCfg<D>;
-  constexpr int NB = C::NB, NSK = C::NSK, NSV = C::NSV;
+  constexpr int NB = C::NB, NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* sQ = smem + C::kQ;
-  uint8_t* sdO = smem + C::kdO;
-  uint8_t* sK = smem + C::kK;
-  uint8_t* sV = smem + C::kV;
+  uint8_t* sKV = smem + C::kKV;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
-  uint64_t* bar_q = bars;              // [2]   Q_x and dO_x landed
-  uint64_t* bar_sp = bars + 2;         // [2]   S_x and dP_x complete
-  uint64_t* bar_ds = bars + 4;         // [2]   dS_x written by its 128 threads
-  uint64_t* bar_acc = bars + 6;        //       every MMA complete
-  uint64_t* bar_kf = bars + 8;         // [NSK]
-  uint64_t* bar_ke = bar_kf + NSK;     // [NSK]
-  uint64_t* bar_vf = bar_ke + NSK;     // [NSV]
-  uint64_t* bar_ve = bar_vf + NSV;     // [NSV]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + 2 * NSK + 2 * NSV);
+  uint64_t* bar_qdo = bars;            //       Q and dO written to tensor memory (256 threads)
+  uint64_t* bar_acc = bars + 1;        //       every MMA complete
+  uint64_t* bar_sp = bars + 2;         // [2]   S and dP of buffer u complete
+  uint64_t* bar_ds = bars + 4;         // [2]   dS of buffer u written by its 128 threads
+  uint64_t* bar_f = bars + 6;          // [NST] stage full
+  uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 2 * NST);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = blockIdx.z;
+  const int b = blockIdx.z, hq = blockIdx.y;
   const int G = p.Hq / p.Hkv;
-  SlotGeom g0, g1;
-  if (p.pair_heads) {
-    const int t = p.T - 1 - int(blockIdx.x);
-    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y), p.cap_pad / kBN);
-    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y) + 1, p.cap_pad / kBN);
-  } else {
-    const int t = p.T - 1 - 2 * int(blockIdx.x);
-    g0 = load_slot(p.tile_meta, b, p.T, t - 1, int(blockIdx.y), p.cap_pad / kBN);
-    g1 = load_slot(p.tile_meta, b, p.T, t, int(blockIdx.y), p.cap_pad / kBN);
-  }
-  const int kv_plane = b * p.Hkv + g1.hq / G;
-  const int ns = max(g0.ns, g1.ns);
-  const int wlo = min(g0.wlo, g1.wlo);
-  const int whi = max(g0.whi, g1.whi);
-  const int n_steps = 2 * (ns + (whi - wlo));  // key half-tiles
+  const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
+  const SlotGeom g = load_slot(p.tile_meta, b, p.T, t, hq, p.cap_pad / kBN);
+  const int kv_plane = b * p.Hkv + hq / G;
+  const int q_plane = b * p.Hq + hq;
+  const int ns = g.ns, wlo = g.wlo;
+  const int n_steps = 2 * (ns + (g.whi - wlo));  // key half-tiles
   // first key row of half-tile s in its tensor (side buffer or K/V)
   auto half_y = [&](int s) -> int {
     const int j = s >> 1;
@@ -160,10 +148,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   };
 
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 128); }
+    mbar_init(bar_qdo, 256);
     mbar_init(bar_acc, 1);
-    for (int i = 0; i < NSK; ++i) { mbar_init(bar_kf + i, 1); mbar_init(bar_ke + i, 1); }
-    for (int i = 0; i < NSV; ++i) { mbar_init(bar_vf + i, 1); mbar_init(bar_ve + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 128); }
+    for (int i = 0; i < NST; ++i) { mbar_init(bar_f + i, 1); mbar_init(bar_e + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -189,158 +177,158 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
-#pragma unroll
-      for (int x = 0; x < 2; ++x) {
-        const SlotGeom& g = x ? g1 : g0;
-        if (g.t >= 0) {
-          mbar_expect_tx(bar_q + x, 2 * C::kTile);
-          for (int nb = 0; nb < NB; ++nb) {
-            tma_load_3d(sQ + x * C::kTile + nb * kTileBlockBytes, &mapQ, bar_q + x, nb * 64,
-                        g.t * kBM, b * p.Hq + g.hq);
-            tma_load_3d(sdO + x * C::kTile + nb * kTileBlockBytes, &mapdO, bar_q + x, nb * 64,
-                        g.t * kBM, b * p.Hq + g.hq);
-          }
-        }
-      }
       for (int s = 0; s < n_steps; ++s) {
         const bool side = (s >> 1) < ns;
         const int y = half_y(s);
-        const int sk = s % NSK, sv = s % NSV;
-        if (s >= NSK) wait(bar_ke + sk, (s / NSK - 1) & 1);
-        mbar_expect_tx(bar_kf + sk, C::kHalf);
-        for (int nb = 0; nb < NB; ++nb)
-          tma_load_3d(sK + sk * C::kHalf + nb * kHalfBlockBytes, side ? &mapKs : &mapK, bar_kf + sk,
+        const int st = s % NST;
+        if (s >= NST) wait(bar_e + st, (s / NST - 1) & 1);
+        mbar_expect_tx(bar_f + st, C::kStage);
+        uint8_t* dst = sKV + st * C::kStage;
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_3d(dst + nb * kHalfBlockBytes, side ? &mapKs : &mapK, bar_f + st, nb * 64, y,
+                      kv_plane);
+          tma_load_3d(dst + C::kHalf + nb * kHalfBlockBytes, side ? &mapVs : &mapV, bar_f + st,
                       nb * 64, y, kv_plane);
-        if (s >= NSV) wait(bar_ve + sv, (s / NSV - 1) & 1);
-        mbar_expect_tx(bar_vf + sv, C::kHalf);
-        for (int nb = 0; nb < NB; ++nb)
-          tma_load_3d(sV + sv * C::kHalf + nb * kHalfBlockBytes, side ? &mapVs : &mapV, bar_vf + sv,
-                      nb * 64, y, kv_plane);
+        }
       }
     } else if (warp == 1 && lane == 0) {
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t q_lo[2] = {desc_lo(smem_u32(sQ), 16), desc_lo(smem_u32(sQ + C::kTile), 16)};
-      const uint32_t do_lo[2] = {desc_lo(smem_u32(sdO), 16), desc_lo(smem_u32(sdO + C::kTile), 16)};
-      const uint32_t k_lo0 = desc_lo(smem_u32(sK), 16);                  // K_h as the K-major B of S
-      const uint32_t kt_lo0 = desc_lo(smem_u32(sK), kHalfBlockBytes);    // K_h as the MN-major B of dQ
-      const uint32_t v_lo0 = desc_lo(smem_u32(sV), 16);
-      int n_dq[2] = {0, 0};
-      bool q_seen[2] = {false, false};
-      for (int s = 0; s <= n_steps; ++s) {
+      const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);                // K_h as K-major B of S
+      const uint32_t kt_lo0 = desc_lo(smem_u32(sKV), kHalfBlockBytes);  // K_h as MN-major B of dQ
+      auto issue_sp = [&](int s) {
+        const int st = s % NST, u = s & 1;
+        wait(bar_f + st, (s / NST) & 1);
+        tc_fence_after();
+        const uint32_t k_lo = k_lo0 + st * (C::kStage >> 4), v_lo = k_lo + (C::kHalf >> 4);
+        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const SlotGeom& g = x ? g1 : g0;
-          const uint32_t tb = tmem + x * C::kSlot;
-          if (s >= 1 && slot_active(g, ns, wlo, (s - 1) >> 1)) {
-            const int sk = (s - 1) % NSK;
-            wait(bar_ds + x, n_dq[x] & 1);
-            tc_fence_after();
-            const uint32_t kt_lo = kt_lo0 + sk * (C::kHalf >> 4);
-            umma_ts_lo(tb + C::kdQ, tb + C::kS, kt_lo, idesc_dq, n_dq[x] > 0);
+        for (int k = 0; k < D / 16; ++k)
+          umma_ts_lo(tb + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kHalfBlockBytes),
+                     idesc_s, k > 0);
 #pragma unroll
-            for (int k = 1; k < 4; ++k)
-              umma_ts_lo(tb + C::kdQ, tb + C::kS + k * 8, kt_lo + mnmajor_step(k), idesc_dq, 1);
-            ++n_dq[x];
-          }
-          if (s < n_steps && slot_active(g, ns, wlo, s >> 1)) {
-            const int sk = s % NSK, sv = s % NSV;
-            if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
-            wait(bar_kf + sk, (s / NSK) & 1);
-            tc_fence_after();
-            const uint32_t k_lo = k_lo0 + sk * (C::kHalf >> 4), v_lo = v_lo0 + sv * (C::kHalf >> 4);
+        for (int k = 0; k < D / 16; ++k)
+          umma_ts_lo(tb + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kHalfBlockBytes),
+                     idesc_s, k > 0);
+        tc_commit(bar_sp + u);
+      };
+      wait(bar_qdo, 0);
+      tc_fence_after();
+      if (n_steps > 0) issue_sp(0);
+      if (n_steps > 1) issue_sp(1);
+      for (int s = 0; s < n_steps; ++s) {
+        const int st = s % NST, u = s & 1;
+        wait(bar_ds + u, (s >> 1) & 1);
+        tc_fence_after();
+        const uint32_t kt_lo = kt_lo0 + st * (C::kStage >> 4);
+        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
+        umma_ts_lo(tmem + C::kdQ, tb + C::kS, kt_lo, idesc_dq, s > 0);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k)
-              umma_ss_lo(tb + C::kS, q_lo[x] + kmajor_step(k, kTileBlockBytes),
-                         k_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
-            wait(bar_vf + sv, (s / NSV) & 1);
-            tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k)
-              umma_ss_lo(tb + C::kdP, do_lo[x] + kmajor_step(k, kTileBlockBytes),
-                         v_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
-            tc_commit(bar_sp + x);
-          }
-        }
-        if (s < n_steps) tc_commit(bar_ve + s % NSV);       // dP MMAs reading V_h(s) are issued
-        if (s >= 1) tc_commit(bar_ke + (s - 1) % NSK);      // S(s-1) and dQ(s-1) MMAs are issued
+        for (int k = 1; k < 4; ++k)
+          umma_ts_lo(tmem + C::kdQ, tb + C::kS + k * 8, kt_lo + mnmajor_step(k), idesc_dq, 1);
+        tc_commit(bar_e + st);
+        if (s + 2 < n_steps) issue_sp(s + 2);
       }
       tc_commit(bar_acc);
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-    // ---------------- dS of slot x ----------------
-    const int x = (warp >= 8) ? 1 : 0;
+    const int u = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;
-    const uint32_t tb = tmem + (uint32_t((warp & 3) * 32) << 16) + x * C::kSlot;
-    const SlotGeom g = x ? g1 : g0;
-    const int t = g.t;
-    if (t >= 0) {
-      const int row = t * kBM + r;
-      const bool row_ok = row < p.L;
-      const int q_plane = b * p.Hq + g.hq;
-      const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-      const float2 st = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
-      const float neg_lse2 = -st.x, delta_i = st.y;
-      const int side_full = g.side_full;
-      int n_done = 0;
-      for (int s = 0; s < n_steps; ++s) {
-        if (!slot_active(g, ns, wlo, s >> 1)) continue;
-        const int j = s >> 1;
-        const bool side = j < ns;
-        int c_lo = 0, c_hi = 64;
-        bool need_mask;
-        if (side) {
-          c_hi = lim_i - half_y(s);
-          need_mask = (j >= side_full);
-        } else {
-          const int key0 = half_y(s);
-          c_hi = row - key0 + 1;
-          c_lo = row - p.n_neighbor + 1 - key0;
-          need_mask = (key0 + 63 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-        }
-        wait(bar_sp + x, n_done & 1);
-        tc_fence_after();
-        uint32_t pk[32];
+    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+    const int row = t * kBM + r;
+    const bool row_ok = row < p.L;
+    // ---------------- Q (warps 4-7) and dO (warps 8-11) rows into tensor memory ----------------
+    {
+      const uint4* src = reinterpret_cast<const uint4*>((u ? dOg : Qg) +
+                                                        (size_t(q_plane) * p.L + row) * D);
+      const uint32_t dst = tmem + lane_base + (u ? C::kdOt : C::kQt);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sv[32], dp[32];
-          tmem_ld32(tb + C::kS + c * 32, sv);
-          tmem_ld32(tb + C::kdP + c * 32, dp);
-          tmem_ld_wait();
+      for (int c = 0; c < D / 64; ++c) {
+        uint32_t w[32];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const uint4 v = row_ok ? src[c * 8 + q] : make_uint4(0, 0, 0, 0);
+          w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+        }
+        tmem_st32(dst + c * 32, w);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar_qdo);
+    }
+    // ---------------- dS of half-tiles s = u, u+2, ... ----------------
+    const uint32_t tb = tmem + lane_base + C::kBuf + u * C::kBufStride;
+    const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
+    const float2 stt = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
+    const float neg_lse2 = -stt.x, delta_i = stt.y;
+    for (int s = u; s < n_steps; s += 2) {
+      const int j = s >> 1;
+      const bool side = j < ns;
+      int c_lo = 0, c_hi = 64;
+      bool need_mask;
+      if (side) {
+        c_hi = lim_i - half_y(s);
+        need_mask = (j >= g.side_full);
+      } else {
+        const int key0 = half_y(s);
+        c_hi = row - key0 + 1;
+        c_lo = row - p.n_neighbor + 1 - key0;
+        need_mask = (key0 + 63 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
+      }
+      wait(bar_sp + u, (s >> 1) & 1);
+      tc_fence_after();
+      uint32_t pk[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t sv[32], dp[32];
+        tmem_ld32(tb + C::kS + c * 32, sv);
+        tmem_ld32(tb + C::kdP + c * 32, dp);
+        tmem_ld_wait();
+        if (need_mask) {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             float ds[2];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int col = c * 32 + e + u;
-              float pr = ex2(fmaf(__uint_as_float(sv[e + u]), p.scale_log2, neg_lse2));
-              if (need_mask && !(col >= c_lo && col < c_hi)) pr = 0.f;
-              ds[u] = pr * (__uint_as_float(dp[e + u]) - delta_i);
+            for (int w = 0; w < 2; ++w) {
+              const int col = c * 32 + e + w;
+              float pr = ex2(fmaf(__uint_as_float(sv[e + w]), p.scale_log2, neg_lse2));
+              pr = (col >= c_lo && col < c_hi) ? pr : 0.f;
+              ds[w] = pr * (__uint_as_float(dp[e + w]) - delta_i);
             }
             pk[c * 16 + (e >> 1)] = pack_bf16(ds[0], ds[1]);
           }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, neg_lse2));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, neg_lse2));
+            pk[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - delta_i),
+                                              p1 * (__uint_as_float(dp[e + 1]) - delta_i));
+          }
         }
-        tmem_st32(tb + C::kS, pk);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(bar_ds + x);
-        ++n_done;
       }
-      wait(bar_acc, 0);
-      tc_fence_after();
+      tmem_st32(tb + C::kS, pk);
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar_ds + u);
+    }
+    // ---------------- epilogue: each warpgroup stores half of the row ----------------
+    wait(bar_acc, 0);
+    tc_fence_after();
+    const uint32_t t_acc = tmem + lane_base + C::kdQ + u * (D / 2);
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t rr[32];
-        tmem_ld32(tb + C::kdQ + c * 32, rr);
-        tmem_ld_wait();
-        if (row_ok) {
-          float v[32];
+    for (int c = 0; c < D / 64; ++c) {
+      uint32_t rr[32];
+      tmem_ld32(t_acc + c * 32, rr);
+      tmem_ld_wait();
+      if (row_ok) {
+        float v[32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
-          store_row_chunk32(p.dQ, (size_t(q_plane) * p.L + row) * D + c * 32, p.grad_fp32, v);
-        }
+        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
+        store_row_chunk32(p.dQ, (size_t(q_plane) * p.L + row) * D + u * (D / 2) + c * 32,
+                          p.grad_fp32, v);
       }
     }
   }
@@ -746,10 +734,9 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        int(DkvCfg<D>::kRequest)));
-  const dim3 grid_dq = p.pair_heads ? dim3(ih.n_tiles, d->Hq / 2, d->B)
-                                    : dim3((ih.n_tiles + 1) / 2, d->Hq, d->B);
-  bwd_dq_kernel<D><<<grid_dq, kBwdThreads, DqCfg<D>::kRequest, stream>>>(mq, mdo, mk_h, mv_h, mks_h,
-                                                                         mvs_h, p);
+  bwd_dq_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
+      mk_h, mv_h, mks_h, mvs_h, static_cast<const __nv_bfloat16*>(Q),
+      static_cast<const __nv_bfloat16*>(dO), p);
   record_event(d, 3, stream);
   bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv * lay.split, d->B), kBwdThreads,
                             DkvCfg<D>::kRequest, stream>>>(mq_h, mdo_h, mks, mvs, p);

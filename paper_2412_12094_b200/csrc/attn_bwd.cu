@@ -148,9 +148,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   };
 
   if (tid == 0) {
-    mbar_init(bar_qdo, 256);
+    mbar_init(bar_qdo, 8);
     mbar_init(bar_acc, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 4); }
     for (int i = 0; i < NST; ++i) { mbar_init(bar_f + i, 1); mbar_init(bar_e + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
@@ -174,7 +174,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   };
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
       for (int s = 0; s < n_steps; ++s) {
@@ -233,7 +233,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tc_commit(bar_acc);
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
     const int u = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
@@ -256,7 +256,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       }
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar_qdo);
+      mbar_arrive_warp(bar_qdo);
     }
     // ---------------- dS of half-tiles s = u, u+2, ... ----------------
     const uint32_t tb = tmem + lane_base + C::kBuf + u * C::kBufStride;
@@ -312,7 +312,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tmem_st32(tb + C::kS, pk);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar_ds + u);
+      mbar_arrive_warp(bar_ds + u);
     }
     // ---------------- epilogue: each warpgroup stores half of the row ----------------
     wait(bar_acc, 0);
@@ -418,8 +418,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   if (tid == 0) {
     mbar_init(bar_kv, 1);
     mbar_init(bar_acc, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_pds + i, 128); }
-    for (int i = 0; i < NSTQ; ++i) { mbar_init(bar_qf + i, 1); mbar_init(bar_qe + i, 1); mbar_init(bar_sf + i, 64); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_pds + i, 4); }
+    for (int i = 0; i < NSTQ; ++i) { mbar_init(bar_qf + i, 1); mbar_init(bar_qe + i, 1); mbar_init(bar_sf + i, 2); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -444,7 +444,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   auto q0_of = [&](int it) { return (qh_lo + it / n_g) * 64; };
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     if (warp == 0 && lane == 0 && n_it > 0) {
       // ---------------- TMA producer ----------------
       mbar_expect_tx(bar_kv, 2 * C::kTile);
@@ -517,11 +517,11 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                                    : make_float2(INFINITY, 0.f);
         if (it >= NSTQ) wait(bar_qe + st, (it / NSTQ - 1) & 1);
         s_stat[st * 64 + i] = make_float2(-v.x, v.y);
-        mbar_arrive(bar_sf + st);
+        mbar_arrive_warp(bar_sf + st);
       }
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
     // ---------------- P^T and dS^T ----------------
     const int u = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;
@@ -552,7 +552,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       wait(bar_sf + st, (it / NSTQ) & 1);
       wait(bar_sp + u, (it >> 1) & 1);
       tc_fence_after();
-      const float2* stat = s_stat + st * 64;
+      // two columns' (-LSE in log2 units, Delta) per shared-memory load
+      const float4* stat2 = reinterpret_cast<const float4*>(s_stat + st * 64);
       uint32_t pkp[32], pkd[32];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
@@ -560,26 +561,36 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tmem_ld32(tb + C::kST + c * 32, sv);
         tmem_ld32(tb + C::kdPT + c * 32, dp);
         tmem_ld_wait();
+        if (need_mask) {
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float pr[2], ds[2];
-#pragma unroll
-          for (int w = 0; w < 2; ++w) {
-            const int col = c * 32 + e + w;
-            const float2 sd = stat[col];  // (-LSE in log2 units, Delta)
-            pr[w] = ex2(fmaf(__uint_as_float(sv[e + w]), p.scale_log2, sd.x));
-            if (need_mask && !(col >= c_lo && col < c_hi)) pr[w] = 0.f;
-            ds[w] = pr[w] * (__uint_as_float(dp[e + w]) - sd.y);
+          for (int e = 0; e < 32; e += 2) {
+            const int col = c * 32 + e;
+            const float4 sd = stat2[col >> 1];
+            float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, sd.x));
+            float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, sd.z));
+            p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
+            p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+            pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
+            pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
+                                               p1 * (__uint_as_float(dp[e + 1]) - sd.w));
           }
-          pkp[c * 16 + (e >> 1)] = pack_bf16(pr[0], pr[1]);
-          pkd[c * 16 + (e >> 1)] = pack_bf16(ds[0], ds[1]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float4 sd = stat2[(c * 32 + e) >> 1];
+            const float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, sd.x));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, sd.z));
+            pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
+            pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
+                                               p1 * (__uint_as_float(dp[e + 1]) - sd.w));
+          }
         }
       }
       tmem_st32(tb + C::kST, pkp);
       tmem_st32(tb + C::kdPT, pkd);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar_pds + u);
+      mbar_arrive_warp(bar_pds + u);
     }
 
     // ---------------- epilogue: warps 4-7 take dV, warps 8-11 take dK ----------------

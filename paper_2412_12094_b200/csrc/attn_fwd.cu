@@ -134,7 +134,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
   uint64_t* bar_q = bars;                   // [2]   Q of slot x landed
   uint64_t* bar_s = bars + 2;               // [2]   S_x complete (and every earlier MMA)
-  uint64_t* bar_p = bars + 4;               // [2]   P_x written by its 128 softmax threads
+  uint64_t* bar_p = bars + 4;               // [2]   P_x written by the 4 softmax warps of slot x
   uint64_t* bar_o = bars + 6;               //       every MMA of the CTA complete
   uint64_t* bar_kf = bars + 8;              // [NST] K stage full
   uint64_t* bar_ke = bar_kf + NST;          // [NST] K stage free
@@ -166,7 +166,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   const int n_tiles = ns + (whi - wlo);
 
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_s + i, 1); mbar_init(bar_p + i, 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_q + i, 1); mbar_init(bar_s + i, 1); mbar_init(bar_p + i, 4); }
     mbar_init(bar_o, 1);
     for (int i = 0; i < NST; ++i) {
       mbar_init(bar_kf + i, 1); mbar_init(bar_ke + i, 1); mbar_init(bar_vf + i, 1); mbar_init(bar_ve + i, 1);
@@ -371,7 +371,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
         tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(bar_p + x);
+        mbar_arrive_warp(bar_p + x);
         ++n_done;
       }
 

@@ -263,7 +263,7 @@ def bench_decode(device, peaks, steps=4096):
     ws = api.alloc_bytes(api.sepllm_decode_workspace_bytes(desc))
     api.sepllm_cache_init(desc, state)
     pool = 256
-    warm = 12000                      # enough tokens to fill the separator cache (s / rho plus slack)
+    warm = 12032                      # enough tokens to fill the separator cache (s / rho plus slack)
     T = warm + steps
     ids = inputs.decode_stream_ids(c["seed"], B, T, c["rho"])
     ids_d = torch.from_numpy(np.ascontiguousarray(ids.T)).to(device)
@@ -271,12 +271,12 @@ def bench_decode(device, peaks, steps=4096):
     o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=device)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=device)
 
-    def step(t):
-        api.sepllm_cache_update(desc, state, Kc, Vc, ids_d[t], inputs.SEP_IDS, kp[t % pool], vp[t % pool])
+    def step(t, ids_row):
+        api.sepllm_cache_update(desc, state, Kc, Vc, ids_row, inputs.SEP_IDS, kp[t % pool], vp[t % pool])
         api.sepllm_decode(desc, 0.0, qp[t % pool], state, Kc, Vc, o, lse, ws)
 
     for t in range(warm):
-        step(t)
+        step(t, ids_d[t])
     torch.cuda.synchronize()
     st0 = api.read_cache_state(state)
     # bookkeeping of Size_run per step (sizes only) for the byte count
@@ -295,10 +295,25 @@ def bench_decode(device, peaks, steps=4096):
                 size_sep[b] = min(c["s"], size_sep[b] + sum(win_flags[b][:n_past]))
                 win_flags[b] = win_flags[b][n_past:]
             rows += size_init[b] + size_sep[b] + len(win_flags[b])
+    # One CUDA graph holds `pool` consecutive steps (4 kernels each); the token ids of a chunk are
+    # copied into the graph's fixed input buffer inside the timed region.
+    assert warm % pool == 0 and steps % pool == 0
+    ids_buf = torch.empty((pool, B), dtype=torch.int32, device=device)
+    ids_buf.copy_(ids_d[warm:warm + pool])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(pool):
+                step(warm + i, ids_buf[i])
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for t in range(warm, T):
-        step(t)
+    for t0 in range(warm, T, pool):
+        ids_buf.copy_(ids_d[t0:t0 + pool], non_blocking=True)
+        graph.replay()
     e1.record()
     torch.cuda.synchronize()
     assert api.sepllm_last_device_status(state) == 0
@@ -350,6 +365,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_long_r10", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / index-stream / e2e / CPU legs")
+    ap.add_argument("--leg", default="all", choices=["all", "decode", "index"],
+                    help="decode / index: run only that secondary leg and print its JSON")
     ap.add_argument("--cpu-prefix", type=int, default=8192)
     ap.add_argument("--cpu-heads", type=int, default=4)
     args = ap.parse_args()
@@ -402,6 +419,9 @@ def main():
             pass
 
     peaks = load_peaks()
+    if args.leg != "all":
+        print(json.dumps(bench_decode(device, peaks) if args.leg == "decode" else bench_index_stream(device, peaks)))
+        return
     wl = Workload(args.workload, rank, device)
     wl.step()
     pairs, side_pairs = wl.kept_pairs()

@@ -220,124 +220,245 @@ cache_update_state(sepllm_cache_header h, uint8_t* __restrict__ state,
 // ---------------------------------------------------------------------------
 constexpr int kDecThreads = 128;
 
+// Ring starts are below the ring size and v is below the region's entry count, so one conditional
+// subtraction wraps the index (no integer division on the decode path).
 __device__ __forceinline__ int virtual_to_slot(int v, const sepllm_cache_seq& q,
                                                const sepllm_cache_desc& d) {
   if (v < q.size_init) return v;
   v -= q.size_init;
-  if (v < q.size_sep) return d.a + (q.sep_start + v) % d.s;
+  if (v < q.size_sep) {
+    const int x = q.sep_start + v;
+    return d.a + (x >= d.s ? x - d.s : x);
+  }
   v -= q.size_sep;
-  return d.a + d.s + (q.win_start + v) % (d.c - d.a);
+  const int ring = d.c - d.a, x = q.win_start + v;
+  return d.a + d.s + (x >= ring ? x - ring : x);
 }
 
-// grid (splits, Hkv, B).  Each warp takes rows of its split in turn; a row of D bf16 is read by
-// D/8 lanes with one 16-byte load each, so a warp covers 32/(D/8) rows per step.  The G query
-// heads sharing the kv head are handled together so K and V are read once.
-template <int D, int G>
+// ---- warp-level MMA pieces used by the decode kernel (bf16 inputs, fp32 accumulation) ----
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+// 16-byte asynchronous copy; src_bytes = 0 writes zeros.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int kDecStages = 3;
+constexpr int kDecTile = 16;  // cache rows per warp tile
+
+template <int D>
+constexpr int decode_smem_bytes() {
+  // per warp: kDecStages x (K tile + V tile); reused after the loop for the warps' partial results
+  return (kDecThreads / 32) * kDecStages * 2 * kDecTile * D * 2;
+}
+
+// grid (splits, Hkv, B), 4 warps.  HBM-bound: the kernel exists to stream every retained K/V row
+// once.  Each warp is an independent flash-decoding worker over its share of the split's rows:
+// 16-row K and V tiles arrive through a 3-stage cp.async ring (virtual entry -> slot mapping done
+// per row; rows past the end are zero-filled), the G query heads of the kv head sit in the M
+// dimension of warp-level MMAs (rows G..15 are zero), scores go through an online softmax with a
+// lazily moved reference, and O accumulates in registers.  The four warps' partials are merged
+// through shared memory into one (m, l, acc) record per (query head, split).
+template <int D>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
              const uint8_t* __restrict__ state, const __nv_bfloat16* __restrict__ Kc,
              const __nv_bfloat16* __restrict__ Vc, float* __restrict__ part_ml,
              float* __restrict__ part_acc, int splits) {
-  constexpr int LPR = D / 8;        // lanes per row
-  constexpr int RPW = 32 / LPR;     // rows per warp step
+  constexpr int CH = D / 8;                 // 16-byte chunks per row
+  constexpr int ROWB = D * 2;               // bytes per row
+  constexpr int TILEB = kDecTile * ROWB;    // bytes of one K (or V) tile
   constexpr int NW = kDecThreads / 32;
+  constexpr int RPP = 32 / CH;              // rows covered by one pass of the warp's copies
+  extern __shared__ __align__(128) uint8_t dec_smem[];
   const sepllm_cache_desc d = h.desc;
+  const int G = d.Hq / d.Hkv;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int sub = lane / LPR, l = lane % LPR;
   CacheView cv = cache_view(const_cast<uint8_t*>(state), h);
   const sepllm_cache_seq sq = cv.seq[b];
   const int size_run = sq.size_init + sq.size_sep + sq.size_win;
-  const int per = (size_run + splits - 1) / splits;
+  const int per = ((size_run + splits - 1) / splits + kDecTile - 1) / kDecTile * kDecTile;
   const int v0 = split * per, v1 = min(size_run, v0 + per);
+  const int n_tiles = (v1 > v0) ? (v1 - v0 + kDecTile - 1) / kDecTile : 0;
+  const int my_n = (n_tiles > wid) ? (n_tiles - wid + NW - 1) / NW : 0;  // tiles wid, wid+NW, ...
 
-  // this lane's 8 elements of each of the G queries, pre-scaled to log2 units
-  float qf[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const uint4 raw = *reinterpret_cast<const uint4*>(
-        q_in + (size_t(b) * d.Hq + hk * G + g) * D + l * 8);
-    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 f2 = __bfloat1622float2(p2[e]);
-      qf[g][2 * e] = f2.x * scale_log2;
-      qf[g][2 * e + 1] = f2.y * scale_log2;
-    }
-  }
-  float m[G], lsum[G], acc[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    m[g] = -INFINITY;
-    lsum[g] = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
-  }
   const size_t plane = (size_t(b) * d.Hkv + hk) * h.slots * D;
-  // Every lane of the warp takes the same number of trips (the shuffles below need all 32
-  // lanes); a sub-row past the end of the split reloads the last row and is not accumulated.
-  for (int base = v0 + wid * RPW; base < v1; base += NW * RPW) {
-    const int vrow = base + sub;
-    const bool valid = vrow < v1;
-    const int slot = virtual_to_slot(valid ? vrow : v1 - 1, sq, d);
-    const uint4 kraw = *reinterpret_cast<const uint4*>(Kc + plane + size_t(slot) * D + l * 8);
-    const uint4 vraw = *reinterpret_cast<const uint4*>(Vc + plane + size_t(slot) * D + l * 8);
-    const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kraw);
-    const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vraw);
-    float kf[8], vf[8];
+  const uint8_t* Kp = reinterpret_cast<const uint8_t*>(Kc + plane);
+  const uint8_t* Vp = reinterpret_cast<const uint8_t*>(Vc + plane);
+  uint8_t* wbase = dec_smem + wid * (kDecStages * 2 * TILEB);
+  const uint32_t wbase_u = smem_u32(wbase);
+
+  // Q fragments (A operand, row = query head of the group): registers 0 and 2 of each k-step
+  const int frow = lane >> 2, fcol = (lane & 3) * 2;
+  uint32_t qa[D / 16][4];
+  {
+    const __nv_bfloat16* qrow = q_in + (size_t(b) * d.Hq + hk * G + min(frow, G - 1)) * D;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 a2 = __bfloat1622float2(k2[e]);
-      const float2 b2 = __bfloat1622float2(v2[e]);
-      kf[2 * e] = a2.x; kf[2 * e + 1] = a2.y;
-      vf[2 * e] = b2.x; vf[2 * e + 1] = b2.y;
+    for (int ks = 0; ks < D / 16; ++ks) {
+      qa[ks][0] = (frow < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + fcol) : 0u;
+      qa[ks][2] = (frow < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + fcol) : 0u;
+      qa[ks][1] = 0u;
+      qa[ks][3] = 0u;
     }
+  }
+
+  // copies of tile `i` (this warp's i-th) into stage i % kDecStages
+  const int crow = lane / CH, cch = lane % CH;
+  auto issue = [&](int i) {
+    const int tile = wid + i * NW;
+    const int vbase = v0 + tile * kDecTile;
+    const uint32_t sK = wbase_u + (i % kDecStages) * 2 * TILEB, sV = sK + TILEB;
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float s = 0.f;
+    for (int pss = 0; pss < kDecTile / RPP; ++pss) {
+      const int r = pss * RPP + crow;
+      const int v = vbase + r;
+      const bool valid = v < v1;
+      const int slot = virtual_to_slot(valid ? v : v1 - 1, sq, d);
+      const uint32_t off = uint32_t(r) * ROWB + (uint32_t(cch ^ (r & 7)) << 4);
+      const size_t goff = size_t(slot) * ROWB + cch * 16;
+      cp_async16(sK + off, Kp + goff, valid ? 16u : 0u);
+      cp_async16(sV + off, Vp + goff, valid ? 16u : 0u);
+    }
+  };
+
+  float oacc[D / 8][4];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) s = fmaf(qf[g][e], kf[e], s);
+  for (int n = 0; n < D / 8; ++n)
 #pragma unroll
-      for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      if (valid) {
-        const float mn = fmaxf(m[g], s);
-        const float corr = ex2(m[g] - mn);
-        const float pexp = ex2(s - mn);
-        m[g] = mn;
-        lsum[g] = lsum[g] * corr + pexp;
+    for (int e = 0; e < 4; ++e) oacc[n][e] = 0.f;
+  float m_ref = -INFINITY, l_part = 0.f;  // of row `frow`; l_part is this lane's share of the sum
+
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(acc[g][e], corr, pexp * vf[e]);
+  for (int s = 0; s < kDecStages - 1; ++s) {
+    if (s < my_n) issue(s);
+    cp_async_commit();
+  }
+  for (int i = 0; i < my_n; ++i) {
+    cp_async_wait<kDecStages - 2>();
+    __syncwarp();
+    if (i + kDecStages - 1 < my_n) issue(i + kDecStages - 1);
+    cp_async_commit();
+
+    const uint32_t sK = wbase_u + (i % kDecStages) * 2 * TILEB, sV = sK + TILEB;
+    // S[16 heads x 16 rows] = Q K^T
+    float sc[2][4];
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[n][e] = 0.f;
+    {
+      const int key = (lane & 7) + ((lane >> 4) << 3);
+      const int chb = (lane >> 3) & 1;
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) {
+        uint32_t kb[4];
+        ldsm_x4(sK + key * ROWB + (uint32_t((2 * ks + chb) ^ (key & 7)) << 4), kb);
+        mma_16816(sc[0], qa[ks], kb[0], kb[1]);
+        mma_16816(sc[1], qa[ks], kb[2], kb[3]);
       }
     }
+    // online softmax over the 16 rows of the tile for query head `frow`
+    const int vbase = v0 + (wid + i * NW) * kDecTile;
+    float sv[4];
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int v = vbase + n * 8 + fcol + e;
+        sv[n * 2 + e] = (v < v1) ? sc[n][e] * scale_log2 : -INFINITY;
+      }
+    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    float corr = 1.f;
+    bool rescale = false;
+    if (mx > m_ref + 8.f) {  // lazy: the reference moves only when the maximum grew by > 2^8
+      corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
+      m_ref = mx;
+      rescale = true;
+    }
+    const float m_eff = (m_ref == -INFINITY) ? 0.f : m_ref;
+    const float p0 = ex2(sv[0] - m_eff), p1 = ex2(sv[1] - m_eff);
+    const float p2 = ex2(sv[2] - m_eff), p3 = ex2(sv[3] - m_eff);
+    l_part = l_part * corr + (p0 + p1) + (p2 + p3);
+    if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+      for (int n = 0; n < D / 8; ++n) { oacc[n][0] *= corr; oacc[n][1] *= corr; }
+    }
+    uint32_t pa[4];
+    pa[0] = pack_bf16(p0, p1);
+    pa[1] = 0u;
+    pa[2] = pack_bf16(p2, p3);
+    pa[3] = 0u;
+    // O[16 heads x D] += P V
+    {
+      const int key = (lane & 7) + (((lane >> 3) & 1) << 3);
+      const int chb = lane >> 4;
+#pragma unroll
+      for (int j = 0; j < CH; j += 2) {
+        uint32_t vb[4];
+        ldsm_x4_trans(sV + key * ROWB + (uint32_t((j + chb) ^ (key & 7)) << 4), vb);
+        mma_16816(oacc[j], pa, vb[0], vb[1]);
+        mma_16816(oacc[j + 1], pa, vb[2], vb[3]);
+      }
+    }
+    __syncwarp();  // every lane is done with this stage before a later copy overwrites it
   }
+  cp_async_wait<0>();
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+  __syncthreads();  // all warps are out of their stage buffers
 
-  // combine the RPW sub-rows of the warp, then the NW warps, through shared memory
-  __shared__ float sm_m[NW * RPW][G];
-  __shared__ float sm_l[NW * RPW][G];
-  __shared__ float sm_acc[NW * RPW][G][D];
-  const int slot_id = wid * RPW + sub;
+  // merge the warps' partials: sm_ml[w][g] = (m, l), sm_acc[w][g][D]
+  float2* sm_ml = reinterpret_cast<float2*>(dec_smem);
+  float* sm_acc = reinterpret_cast<float*>(dec_smem + NW * 8 * sizeof(float2));
+  if (frow < G) {
+    if ((lane & 3) == 0) sm_ml[wid * 8 + frow] = make_float2(m_ref, l_part);
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    if (l == 0) { sm_m[slot_id][g] = m[g]; sm_l[slot_id][g] = lsum[g]; }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) sm_acc[slot_id][g][l * 8 + e] = acc[g][e];
+    for (int n = 0; n < D / 8; ++n)
+      *reinterpret_cast<float2*>(sm_acc + (wid * 8 + frow) * D + n * 8 + fcol) =
+          make_float2(oacc[n][0], oacc[n][1]);
   }
   __syncthreads();
   for (int idx = tid; idx < G * D; idx += kDecThreads) {
     const int g = idx / D, e = idx % D;
     float mm = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < NW * RPW; ++r) mm = fmaxf(mm, sm_m[r][g]);
+    for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sm_ml[w * 8 + g].x);
     float ll = 0.f, aa = 0.f;
 #pragma unroll
-    for (int r = 0; r < NW * RPW; ++r) {
-      const float sc = (sm_m[r][g] == -INFINITY) ? 0.f : ex2(sm_m[r][g] - mm);
-      ll += sm_l[r][g] * sc;
-      aa += sm_acc[r][g][e] * sc;
+    for (int w = 0; w < NW; ++w) {
+      const float2 ml = sm_ml[w * 8 + g];
+      const float scf = (ml.x == -INFINITY) ? 0.f : ex2(ml.x - mm);
+      ll += ml.y * scf;
+      aa += sm_acc[(w * 8 + g) * D + e] * scf;
     }
-    const size_t u = ((size_t(b) * d.Hq + hk * G + g) * splits + split);
-    part_acc[u * D + e] = aa;
-    if (e == 0) { part_ml[u * 2] = mm; part_ml[u * 2 + 1] = ll; }
+    const size_t uo = ((size_t(b) * d.Hq + hk * G + g) * splits + split);
+    part_acc[uo * D + e] = aa;
+    if (e == 0) { part_ml[uo * 2] = mm; part_ml[uo * 2 + 1] = ll; }
   }
 }
 
@@ -363,10 +484,10 @@ __global__ void decode_combine(sepllm_cache_header h, const float* __restrict__ 
 }
 
 static int decode_splits(const sepllm_cache_desc* d) {
-  // enough CTAs for several per SM, at least ~128 rows each
+  // about four CTAs per SM over the whole grid, each with at least 256 rows (64 per warp)
   const int units = d->B * d->Hkv;
-  int s = (148 * 8 + units - 1) / units;
-  const int max_by_rows = (d->c + 127) / 128;
+  int s = (148 * 4 + units - 1) / units;
+  const int max_by_rows = (d->c + 255) / 256;
   if (s > max_by_rows) s = max_by_rows;
   if (s < 1) s = 1;
   if (s > 64) s = 64;
@@ -452,14 +573,18 @@ extern "C" sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* 
   return SEPLLM_OK;
 }
 
-template <int D, int G>
-static void launch_decode(const sepllm_cache_header& h, float scale_log2, const void* q,
-                          const void* state, const void* Kc, const void* Vc, float* ml, float* acc,
-                          int splits, cudaStream_t stream) {
-  decode_split<D, G><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, 0, stream>>>(
+template <int D>
+static sepllm_status launch_decode(const sepllm_cache_header& h, float scale_log2, const void* q,
+                                   const void* state, const void* Kc, const void* Vc, float* ml,
+                                   float* acc, int splits, cudaStream_t stream) {
+  constexpr int smem = decode_smem_bytes<D>();
+  static_assert(smem >= (kDecThreads / 32) * 8 * (8 + D * 4), "partials fit in the stage buffers");
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem));
+  decode_split<D><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
       h, scale_log2, static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(state),
-      static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc,
-      splits);
+      static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc, splits);
+  return SEPLLM_OK;
 }
 
 extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const void* q,
@@ -481,15 +606,11 @@ extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scal
   float* acc = reinterpret_cast<float*>(ws + kAlign + align_up(units * 2 * sizeof(float)));
   if (scale == 0.f) scale = 1.0f / sqrtf(float(desc->d));
   const float scale_log2 = scale * 1.4426950408889634f;
-  const int G = desc->Hq / desc->Hkv;
-#define SEPLLM_DEC(DD, GG)                                                                      \
-  if (desc->d == DD && G == GG) {                                                               \
-    launch_decode<DD, GG>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, stream);           \
-  } else
-  SEPLLM_DEC(128, 1) SEPLLM_DEC(128, 2) SEPLLM_DEC(128, 4) SEPLLM_DEC(128, 8)
-  SEPLLM_DEC(64, 1) SEPLLM_DEC(64, 2) SEPLLM_DEC(64, 4) SEPLLM_DEC(64, 8)
-  { return SEPLLM_UNSUPPORTED; }
-#undef SEPLLM_DEC
+  if (desc->d == 128)
+    st = launch_decode<128>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, stream);
+  else
+    st = launch_decode<64>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, stream);
+  if (st != SEPLLM_OK) return st;
   if (desc->d == 128)
     decode_combine<128><<<dim3(desc->Hq, desc->B), 128, 0, stream>>>(
         h, ml, acc, splits, static_cast<__nv_bfloat16*>(o), lse);

@@ -137,18 +137,20 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
  * callback that runs where cudaMalloc is forbidden, or a latency-critical loop
  * that must not take cudaMalloc's device-wide synchronisation.  (The paper has
  * no counterpart; this is a packaging variant of the index build.)
- * The scratch lives in a fixed 256 KB array inside the library image, present
- * on every device that loads the library until the process exits.  Limit:
- * B * ceil(L / 4096) <= 65536 chunks; beyond it the call returns
- * SEPLLM_BUFFER_TOO_SMALL and launches nothing.  The call itself allocates
+ * The scratch lives in a fixed 256 KB array (65536 words) inside the library
+ * image, present on every device that loads the library until the process
+ * exits.  A call needs two words per 4096-token chunk plus one per sequence,
+ * so the limit is B * (2 * ceil(L / 4096) + 1) <= 65536 (for example 32
+ * sequences of 4 M ids); beyond it the call returns SEPLLM_BUFFER_TOO_SMALL
+ * and launches nothing.  The call itself allocates
  * nothing (no cudaMalloc / cudaFree, no allocating library routine).
  * The first call on each device looks up the array's device address; make that
  * first call outside any stream capture.  All calls on a device share the one
  * array: two calls whose kernels may overlap on the GPU (different streams
  * without ordering, or different host threads) race on it and must be
- * serialised by the caller.  Nothing in the array has to be zero on entry: every
- * word a call reads it has written itself, so back-to-back calls are
- * independent.  Other arguments and the written index are exactly those of
+ * serialised by the caller.  The array keeps the last call's contents; each
+ * call clears the words it is going to use (a memset on `stream`, before its
+ * kernels), so back-to-back calls are independent.  Other arguments and the written index are exactly those of
  * sepllm_build_index. */
 sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* sep_ids, void* index, void* stream);

@@ -138,7 +138,7 @@ def sepllm_build_index(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index:
 
 def sepllm_build_index_static(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index: torch.Tensor):
     """Index build for callers that cannot allocate a scratch buffer: the library's own fixed
-    array is used instead (B * ceil(L/4096) <= 65536).  Calls that may overlap on the GPU must be
+    array is used instead (B * (2 * ceil(L/4096) + 1) <= 65536).  Calls that may overlap on the GPU must be
     serialised by the caller; make the first call on a device outside any stream capture."""
     arr, p, n = _sep_array(sep_ids)
     assert n == desc.n_sep

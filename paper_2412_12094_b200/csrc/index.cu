@@ -1,11 +1,16 @@
 // Separator index builder: token ids -> cnt / lim / side_pos / n_side / tile_meta.
 //
 // The mask of Eq. 2 depends on token ids only, so one index serves every head and
-// layer.  Three launches, none of which waits on another block:
-//   1. index_count : side-member count of every 4096-token chunk
-//   2. index_scan  : chunk offset (sum of earlier chunk counts) + in-chunk prefix scan;
-//                    writes cnt, the shifted copy lim[i] = cnt[i-n+1], and side_pos
-//   3. index_tiles : per query tile metadata, side_pos tail fill, header
+// layer.  The token ids are read once:
+//   index_scan  : one block per 4096-token chunk.  Flags, block-local prefix counts, and a
+//                 decoupled look-back over the earlier chunks' published totals give every
+//                 position its global count; the block writes cnt, the shifted copy
+//                 lim[i] = cnt[i-n+1], side_pos, and adds its rows' lim values to the kept-pair
+//                 count of the query tiles they fall in.
+//   index_tiles : per query tile metadata from lim's two end rows, closed-form window pairs,
+//                 side_pos tail fill, header.
+// Chunks are handed out by an atomic ticket per sequence, so a block only ever waits on blocks
+// that started before it; the wait is bounded all the same.
 #include <mutex>
 
 #include "common.cuh"
@@ -22,67 +27,81 @@ __device__ __forceinline__ int warp_sum(int v) {
   return v;
 }
 
-__device__ __forceinline__ int block_sum(int v, int* warp_buf) {
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  v = warp_sum(v);
-  if (lane == 0) warp_buf[wid] = v;
-  __syncthreads();
-  int t = (lane < (blockDim.x >> 5)) ? warp_buf[lane] : 0;
-  t = warp_sum(t);
-  __syncthreads();
-  return t;
+// Membership among the first NS entries of the list (the host pads the list with copies of its
+// first id, so NS may exceed the real count).
+template <int NS>
+__device__ __forceinline__ bool in_sep_list(int32_t tok, const SepIds& s) {
+  bool f = false;
+#pragma unroll
+  for (int k = 0; k < NS; ++k) f |= (tok == s.id[k]);
+  return f;
 }
 
-__global__ void __launch_bounds__(kIdxThreads)
-index_count(const int32_t* __restrict__ token_ids, int L, int n_init, SepIds sep,
-            int32_t* __restrict__ chunk_sums, int n_chunks) {
-  __shared__ int warp_buf[32];
-  const int b = blockIdx.y, chunk = blockIdx.x;
-  const int32_t* ids = token_ids + static_cast<size_t>(b) * L;
-  const int base = chunk * kIdxChunk;
-  int c = 0;
-#pragma unroll 4
-  for (int k = 0; k < kIdxPerThread; ++k) {
-    const int j = base + k * kIdxThreads + threadIdx.x;
-    if (j < L) c += (j < n_init) || is_separator(ids[j], sep);
-  }
-  c = block_sum(c, warp_buf);
-  if (threadIdx.x == 0) chunk_sums[b * n_chunks + chunk] = c;
+// Scratch words per call: one 64-bit chunk record (state << 32 | count) per chunk, then one
+// ticket counter per sequence.  Zeroed before the scan kernel runs.
+constexpr uint32_t kChunkAggregate = 1, kChunkPrefix = 2;
+inline size_t index_scratch_words(int B, int n_chunks) {
+  return 2 * size_t(B) * n_chunks + size_t(B);
 }
 
+__device__ __forceinline__ unsigned long long ld_chunk_state(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_chunk_state(unsigned long long* p, uint32_t state, int count) {
+  const unsigned long long v = (static_cast<unsigned long long>(state) << 32) | uint32_t(count);
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+constexpr int kLookbackSpins = 1 << 22;
+constexpr int kMaxTilesPerChunk = kIdxChunk / kIdxPerThread + 2;  // query tiles of >= 16 rows under one chunk
+
+template <int NS>
 __global__ void __launch_bounds__(kIdxThreads)
 index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neighbor, SepIds sep,
-           const int32_t* __restrict__ chunk_sums, int n_chunks, int side_cap,
-           int32_t* __restrict__ cnt, int32_t* __restrict__ lim, int32_t* __restrict__ side_pos,
-           int32_t* __restrict__ n_side, int32_t* status) {
-  __shared__ int warp_buf[32];
-  __shared__ uint8_t flag_s[kIdxChunk];
-  __shared__ int32_t cnt_s[kIdxChunk];
-  const int b = blockIdx.y, chunk = blockIdx.x;
+           unsigned long long* __restrict__ chunk_state, int32_t* __restrict__ tickets,
+           int n_chunks, int side_cap, int32_t* __restrict__ cnt, int32_t* __restrict__ lim,
+           int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
+           int32_t* __restrict__ tile_meta, int T, int BM, int32_t* status) {
+  __shared__ int warp_buf[kIdxThreads / 32];
+  __shared__ int s_chunk, s_off;
+  // counts of the chunk, one pad word per 32 so that a thread's 16 consecutive words and a
+  // warp's 32 consecutive words are both conflict-free
+  __shared__ int32_t cnt_s[kIdxChunk + kIdxChunk / 32];
+  __shared__ int32_t tile_part[kMaxTilesPerChunk];
+  const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) s_chunk = atomicAdd(&tickets[b], 1);
+  __syncthreads();
+  const int chunk = s_chunk;
+  if (chunk >= n_chunks) return;
   const int32_t* ids = token_ids + static_cast<size_t>(b) * L;
   const int base = chunk * kIdxChunk;
 
-  // side members before this chunk
-  int off = 0;
-  for (int k = tid; k < chunk; k += kIdxThreads) off += chunk_sums[b * n_chunks + k];
-  off = block_sum(off, warp_buf);
-
-  // flags, loaded coalesced
-#pragma unroll 4
-  for (int k = 0; k < kIdxPerThread; ++k) {
-    const int p = k * kIdxThreads + tid;
-    const int j = base + p;
-    flag_s[p] = (j < L) ? uint8_t((j < n_init) || is_separator(ids[j], sep)) : uint8_t(0);
-  }
-  __syncthreads();
-
-  // each thread owns 16 consecutive positions
-  uint8_t fl[kIdxPerThread];
-  *reinterpret_cast<uint4*>(fl) = *reinterpret_cast<const uint4*>(&flag_s[tid * kIdxPerThread]);
-  int local = 0;
+  // flags of this thread's 16 consecutive positions
+  const int p0 = tid * kIdxPerThread, j0 = base + p0;
+  uint32_t fl = 0;
+  if (j0 + kIdxPerThread <= L && (reinterpret_cast<uintptr_t>(ids + j0) & 15) == 0) {
+    const int4* src = reinterpret_cast<const int4*>(ids + j0);
 #pragma unroll
-  for (int k = 0; k < kIdxPerThread; ++k) local += fl[k];
+    for (int q = 0; q < 4; ++q) {
+      const int4 v = src[q];
+      fl |= uint32_t(in_sep_list<NS>(v.x, sep)) << (4 * q);
+      fl |= uint32_t(in_sep_list<NS>(v.y, sep)) << (4 * q + 1);
+      fl |= uint32_t(in_sep_list<NS>(v.z, sep)) << (4 * q + 2);
+      fl |= uint32_t(in_sep_list<NS>(v.w, sep)) << (4 * q + 3);
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < kIdxPerThread; ++k)
+      if (j0 + k < L) fl |= uint32_t(in_sep_list<NS>(ids[j0 + k], sep)) << k;
+  }
+  if (j0 < n_init) {  // initial tokens are side members too
+    const int m = max(0, min(kIdxPerThread, min(n_init, L) - j0));
+    fl |= (1u << m) - 1u;
+  }
+  const int local = __popc(fl);
 
   // exclusive scan of `local` over the block
   int incl = local;
@@ -93,42 +112,157 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   }
   if (lane == 31) warp_buf[wid] = incl;
   __syncthreads();
-  int warp_off = 0;
-  for (int k = 0; k < wid; ++k) warp_off += warp_buf[k];
-  int run = off + warp_off + incl - local;
-
-  int32_t* sp = side_pos + static_cast<size_t>(b) * side_cap;
+  int warp_off = 0, total = 0;
 #pragma unroll
-  for (int k = 0; k < kIdxPerThread; ++k) {
-    const int p = tid * kIdxPerThread + k;
-    cnt_s[p] = run;
-    if (fl[k]) {
-      if (run < side_cap) sp[run] = base + p;
+  for (int k = 0; k < kIdxThreads / 32; ++k) {
+    if (k < wid) warp_off += warp_buf[k];
+    total += warp_buf[k];
+  }
+
+  // Chunk-relative counts go to shared memory while warp 0 looks back over the earlier chunks of
+  // the sequence for the number of side members before this chunk.
+  if (wid == 0) {
+    unsigned long long* st = chunk_state + static_cast<size_t>(b) * n_chunks;
+    int off = 0;
+    if (chunk > 0) {
+      if (lane == 0) st_chunk_state(st + chunk, kChunkAggregate, total);
+      int look = chunk - 1;
+      int spins = 0;
+      bool gave_up = false;
+      while (look >= 0) {
+        const int c = look - lane;
+        unsigned long long v = (c >= 0) ? ld_chunk_state(st + c)
+                                        : (static_cast<unsigned long long>(kChunkPrefix) << 32);
+        const uint32_t state = uint32_t(v >> 32);
+        if (__any_sync(0xffffffffu, state == 0)) {  // a predecessor has not published yet
+          if (++spins > kLookbackSpins) { gave_up = true; break; }
+          __nanosleep(64);
+          continue;
+        }
+        const uint32_t prefix_mask = __ballot_sync(0xffffffffu, state == kChunkPrefix);
+        const int first = prefix_mask ? __ffs(prefix_mask) - 1 : 32;  // nearest chunk holding a prefix
+        off += warp_sum((lane <= first) ? int(uint32_t(v)) : 0);
+        if (prefix_mask) break;
+        look -= 32;
+      }
+      if (gave_up && lane == 0) set_status(status, SEPLLM_TIMEOUT);
+    }
+    if (lane == 0) {
+      st_chunk_state(st + chunk, kChunkPrefix, off + total);
+      s_off = off;
+    }
+  }
+  // Position p of the chunk is the lim of row base + shift + p; with BM >= 16 a thread's 16 rows
+  // lie in at most two query tiles, whose side-pair sums are gathered in shared memory.
+  const int shift = n_neighbor - 1;
+  const long long row_lo = static_cast<long long>(base) + shift;
+  const int n_rows = int(max(0LL, min(static_cast<long long>(L) - row_lo,
+                                      static_cast<long long>(min(kIdxChunk, L - base)))));
+  const int t_first = int(row_lo / BM);
+  const bool fast_pairs = (BM >= kIdxPerThread) && (kIdxChunk / BM + 2 <= kMaxTilesPerChunk);
+  for (int k = tid; k < kMaxTilesPerChunk; k += kIdxThreads) tile_part[k] = 0;
+  __syncthreads();
+  {
+    int rel = warp_off + incl - local;
+    const int kb = BM - int((row_lo + p0) % BM);  // rows k >= kb belong to the next tile
+    int s0 = 0, s1 = 0;
+#pragma unroll
+    for (int k = 0; k < kIdxPerThread; ++k) {
+      const int p = p0 + k;
+      cnt_s[p + (p >> 5)] = rel;
+      const int vv = (p < n_rows) ? rel : 0;
+      s0 += (k < kb) ? vv : 0;
+      s1 += (k < kb) ? 0 : vv;
+      rel += (fl >> k) & 1u;
+    }
+    if (fast_pairs) {
+      const int tl = int((row_lo + p0) / BM) - t_first;
+      if (s0) atomicAdd(&tile_part[tl], s0);
+      if (s1) atomicAdd(&tile_part[tl + 1], s1);
+    }
+  }
+  __syncthreads();
+  const int off = s_off;
+
+  // positions of this thread's side members
+  {
+    int32_t* sp = side_pos + static_cast<size_t>(b) * side_cap;
+    int run = off + warp_off + incl - local;
+    uint32_t rest = fl;
+    while (rest) {
+      const int k = __ffs(rest) - 1;
+      rest &= rest - 1;
+      if (run < side_cap) sp[run] = j0 + k;
       else set_status(status, SEPLLM_CAPACITY_EXCEEDED);
       ++run;
     }
   }
-  __syncthreads();
 
   int32_t* cnt_b = cnt + static_cast<size_t>(b) * (L + 1);
   int32_t* lim_b = lim + static_cast<size_t>(b) * L;
-  const int shift = n_neighbor - 1;
+  if (base + kIdxChunk + shift <= L && base >= shift) {  // whole chunk inside both arrays
+    int32_t* cdst = cnt_b + base + tid;
+    int32_t* ldst = lim_b + base + shift + tid;
+#pragma unroll
+    for (int k = 0; k < kIdxPerThread; ++k) {
+      const int p = k * kIdxThreads + tid;
+      const int v = cnt_s[p + (p >> 5)] + off;
+      cdst[k * kIdxThreads] = v;
+      ldst[k * kIdxThreads] = v;
+    }
+  } else {
 #pragma unroll 4
-  for (int k = 0; k < kIdxPerThread; ++k) {
-    const int p = k * kIdxThreads + tid;
-    const int j = base + p;
-    if (j < L) {
-      const int v = cnt_s[p];
-      cnt_b[j] = v;
-      // lim[i] = cnt[max(0, i-n+1)]: zero for i < n-1, else cnt shifted by n-1
-      if (j < shift) lim_b[j] = 0;
-      if (static_cast<long long>(j) + shift < L) lim_b[j + shift] = v;
+    for (int k = 0; k < kIdxPerThread; ++k) {
+      const int p = k * kIdxThreads + tid;
+      const int j = base + p;
+      if (j < L) {
+        const int v = cnt_s[p + (p >> 5)] + off;
+        cnt_b[j] = v;
+        // lim[i] = cnt[max(0, i-n+1)]: zero for i < n-1, else cnt shifted by n-1
+        if (j < shift) lim_b[j] = 0;
+        if (static_cast<long long>(j) + shift < L) lim_b[j + shift] = v;
+      }
     }
   }
-  if (chunk == n_chunks - 1 && tid == kIdxThreads - 1) {
-    cnt_b[L] = run;  // the last thread's running count is the total
-    n_side[b] = run;
+  // side pairs of the query tiles under this chunk's rows: relative sums plus off per row
+  if (n_rows > 0) {
+    int32_t* meta_b = tile_meta + static_cast<size_t>(b) * T * 8;
+    const long long row_hi = row_lo + n_rows;  // exclusive
+    const int t_last = int((row_hi - 1) / BM);
+    if (fast_pairs) {
+      for (int t = t_first + tid; t <= t_last; t += kIdxThreads) {
+        const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
+        const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
+        const int sum = tile_part[t - t_first] + off * int(r1 - r0);
+        if (sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
+      }
+    } else {
+      for (int t = t_first + wid; t <= t_last; t += kIdxThreads / 32) {
+        const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
+        const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
+        int sum = 0;
+        for (long long r = r0 + lane; r < r1; r += 32) {
+          const int p = int(r - row_lo);
+          sum += cnt_s[p + (p >> 5)] + off;
+        }
+        sum = warp_sum(sum);
+        if (lane == 0 && sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
+      }
+    }
   }
+  if (chunk == n_chunks - 1 && tid == 0) {
+    cnt_b[L] = off + total;
+    n_side[b] = off + total;
+  }
+}
+
+// Sum of min(i + 1, n) over rows r0..r1.
+__device__ __forceinline__ long long window_pairs(int r0, int r1, int n) {
+  const long long a = r0 + 1LL, bb = r1 + 1LL;
+  const long long k = min(bb, static_cast<long long>(n));
+  const long long ramp = (a <= k) ? (a + k) * (k - a + 1) / 2 : 0;
+  const long long flat = max(0LL, bb - max(a - 1, static_cast<long long>(n)));
+  return ramp + flat * n;
 }
 
 __global__ void __launch_bounds__(256)
@@ -139,12 +273,10 @@ index_tiles(sepllm_index_header hdr, uint8_t* __restrict__ index) {
   const int32_t* n_side = reinterpret_cast<const int32_t*>(index + hdr.off_n_side);
   int32_t* side_pos = reinterpret_cast<int32_t*>(index + hdr.off_side_pos);
   int32_t* tile_meta = reinterpret_cast<int32_t*>(index + hdr.off_tile_meta);
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
-  const int gw = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-  const int n_warps = gridDim.x * warps_per_block;
+  const int gt = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_threads = gridDim.x * blockDim.x;
 
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
+  if (gt == 0) {
     // everything but the status word, which the scan kernel may have set
     sepllm_index_header* out = reinterpret_cast<sepllm_index_header*>(index);
     const int32_t st = out->status;
@@ -152,31 +284,21 @@ index_tiles(sepllm_index_header hdr, uint8_t* __restrict__ index) {
     out->status = st;
   }
 
-  for (int u = gw; u < B * T; u += n_warps) {
-    const int b = u / T, t = u % T;
+  // one thread per query tile; word 6 already holds the tile's side pairs
+  for (long long u = gt; u < static_cast<long long>(B) * T; u += n_threads) {
+    const int b = int(u / T), t = int(u % T);
     const int32_t* lim_b = lim + static_cast<size_t>(b) * L;
     const int r0 = t * BM;
     const int r1 = min(L, (t + 1) * BM) - 1;
-    int pairs = 0;
-    for (int i = r0 + lane; i <= r1; i += 32) pairs += lim_b[i] + min(i + 1, n);
-    pairs = warp_sum(pairs);
-    if (lane == 0) {
-      int32_t* m = tile_meta + (static_cast<size_t>(b) * T + t) * 8;
-      const int win_lo = max(0, r0 - n + 1), win_hi = r1 + 1;
-      m[0] = lim_b[r0] / BN;
-      m[1] = (lim_b[r1] + BN - 1) / BN;
-      m[2] = win_lo;
-      m[3] = win_hi;
-      m[4] = win_lo / BN;
-      m[5] = (win_hi + BN - 1) / BN;
-      m[6] = pairs;
-      m[7] = 0;
-    }
+    int32_t* m = tile_meta + static_cast<size_t>(u) * 8;
+    const int win_lo = max(0, r0 - n + 1), win_hi = r1 + 1;
+    const int side_pairs = m[6];
+    *reinterpret_cast<int4*>(m) = make_int4(lim_b[r0] / BN, (lim_b[r1] + BN - 1) / BN, win_lo, win_hi);
+    *reinterpret_cast<int4*>(m + 4) = make_int4(win_lo / BN, (win_hi + BN - 1) / BN,
+                                                side_pairs + int(window_pairs(r0, r1, n)), 0);
   }
 
   // side_pos beyond n_side reads -1
-  const int gt = blockIdx.x * blockDim.x + threadIdx.x;
-  const int n_threads = gridDim.x * blockDim.x;
   for (int b = 0; b < B; ++b) {
     const int ns = min(n_side[b], side_cap);
     for (int r = ns + gt; r < side_cap; r += n_threads)
@@ -222,6 +344,46 @@ using namespace sepllm;
 
 static_assert(sizeof(sepllm_index_header) == 256, "index header is 256 bytes");
 
+// Launches shared by the two entry points.  `scratch` holds index_scratch_words() int32 words.
+static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_index_header& h,
+                                  const int32_t* token_ids, const int32_t* sep_ids, uint8_t* blob,
+                                  int32_t* scratch, cudaStream_t stream) {
+  SepIds sep;
+  sep.n = desc->n_sep;
+  for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k)
+    sep.id[k] = (sep.n > 0) ? sep_ids[(k < sep.n) ? k : 0] : -1;
+  const int n_chunks = (desc->L + kIdxChunk - 1) / kIdxChunk;
+  const size_t words = index_scratch_words(desc->B, n_chunks);
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(blob, 0, sizeof(sepllm_index_header), stream));
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(scratch, 0, words * sizeof(int32_t), stream));
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(blob + h.off_tile_meta, 0,
+                                  sizeof(int32_t) * size_t(desc->B) * h.n_tiles * 8, stream));
+  unsigned long long* chunk_state = reinterpret_cast<unsigned long long*>(scratch);
+  int32_t* tickets = scratch + 2 * size_t(desc->B) * n_chunks;
+  dim3 grid(n_chunks, desc->B);
+#define SEPLLM_SCAN(NS)                                                                          \
+  index_scan<NS><<<grid, kIdxThreads, 0, stream>>>(                                              \
+      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, chunk_state, tickets, n_chunks,   \
+      desc->side_cap, reinterpret_cast<int32_t*>(blob + h.off_cnt),                              \
+      reinterpret_cast<int32_t*>(blob + h.off_lim),                                              \
+      reinterpret_cast<int32_t*>(blob + h.off_side_pos),                                         \
+      reinterpret_cast<int32_t*>(blob + h.off_n_side),                                           \
+      reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM,                   \
+      reinterpret_cast<int32_t*>(blob))
+  if (sep.n == 0) SEPLLM_SCAN(0);
+  else if (sep.n <= 8) SEPLLM_SCAN(8);
+  else if (sep.n <= 12) SEPLLM_SCAN(12);
+  else if (sep.n <= 16) SEPLLM_SCAN(16);
+  else if (sep.n <= 32) SEPLLM_SCAN(32);
+  else SEPLLM_SCAN(64);
+#undef SEPLLM_SCAN
+  const long long units = static_cast<long long>(desc->B) * h.n_tiles;
+  const int blocks = int(max(1LL, min(148LL * 8, (units + 255) / 256)));
+  index_tiles<<<blocks, 256, 0, stream>>>(h, blob);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  return SEPLLM_OK;
+}
+
 extern "C" sepllm_status sepllm_index_bytes(const sepllm_index_desc* desc, size_t* index_bytes,
                                             size_t* scratch_bytes) {
   sepllm_index_header h;
@@ -229,7 +391,7 @@ extern "C" sepllm_status sepllm_index_bytes(const sepllm_index_desc* desc, size_
   if (st != SEPLLM_OK) return st;
   if (index_bytes) *index_bytes = size_t(h.total_bytes);
   const int n_chunks = (desc->L + kIdxChunk - 1) / kIdxChunk;
-  if (scratch_bytes) *scratch_bytes = align_up(sizeof(int32_t) * size_t(desc->B) * n_chunks);
+  if (scratch_bytes) *scratch_bytes = align_up(sizeof(int32_t) * index_scratch_words(desc->B, n_chunks));
   return SEPLLM_OK;
 }
 
@@ -243,38 +405,18 @@ extern "C" sepllm_status sepllm_build_index(const sepllm_index_desc* desc,
   if (!aligned(index, kAlign) || !aligned(scratch, kAlign) || !aligned(token_ids, 4))
     return SEPLLM_INVALID_ARG;
   if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  SepIds sep;
-  sep.n = desc->n_sep;
-  for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k) sep.id[k] = (k < sep.n) ? sep_ids[k] : -1;
-
-  uint8_t* blob = static_cast<uint8_t*>(index);
-  const int n_chunks = (desc->L + kIdxChunk - 1) / kIdxChunk;
-  int32_t* chunk_sums = static_cast<int32_t*>(scratch);
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(blob, 0, sizeof(sepllm_index_header), stream));
-  dim3 grid(n_chunks, desc->B);
-  index_count<<<grid, kIdxThreads, 0, stream>>>(token_ids, desc->L, desc->n_init, sep, chunk_sums,
-                                                n_chunks);
-  index_scan<<<grid, kIdxThreads, 0, stream>>>(
-      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, chunk_sums, n_chunks,
-      desc->side_cap, reinterpret_cast<int32_t*>(blob + h.off_cnt),
-      reinterpret_cast<int32_t*>(blob + h.off_lim),
-      reinterpret_cast<int32_t*>(blob + h.off_side_pos),
-      reinterpret_cast<int32_t*>(blob + h.off_n_side), reinterpret_cast<int32_t*>(blob));
-  const int units = desc->B * h.n_tiles;
-  const int blocks = max(1, min(148 * 4, (units + 7) / 8));
-  index_tiles<<<blocks, 256, 0, stream>>>(h, blob);
-  SEPLLM_CUDA_TRY(cudaGetLastError());
-  return SEPLLM_OK;
+  return launch_index(desc, h, token_ids, sep_ids, static_cast<uint8_t*>(index),
+                      static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream_));
 }
 
 // ---------------------------------------------------------------------------
 // Index build without caller-provided scratch
 // ---------------------------------------------------------------------------
-// Chunk sums for sepllm_build_index_static live in this fixed array instead of a caller buffer.
-// 65536 chunks of 4096 ids = 256 KB, held by every device that loads the library until exit.
-constexpr int kStaticChunks = 65536;
-static __device__ __align__(256) int32_t g_static_chunk_sums[kStaticChunks];
+// The scan's chunk records and tickets for sepllm_build_index_static live in this fixed array
+// instead of a caller buffer: 65536 words = 256 KB, held by every device that loads the library
+// until exit.  A call needs 2 words per 4096-token chunk plus one per sequence.
+constexpr int kStaticWords = 65536;
+static __device__ __align__(256) int32_t g_static_chunk_sums[kStaticWords];
 
 constexpr int kMaxDevices = 64;
 static std::mutex g_static_mu;
@@ -308,29 +450,11 @@ extern "C" sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc
   if (!aligned(index, kAlign) || !aligned(token_ids, 4)) return SEPLLM_INVALID_ARG;
   if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
   const int n_chunks = (desc->L + kIdxChunk - 1) / kIdxChunk;
-  if (static_cast<int64_t>(desc->B) * n_chunks > kStaticChunks) return SEPLLM_BUFFER_TOO_SMALL;
-  int32_t* chunk_sums = nullptr;
-  if ((st = static_chunk_sums(&chunk_sums)) != SEPLLM_OK) return st;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  SepIds sep;
-  sep.n = desc->n_sep;
-  for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k) sep.id[k] = (k < sep.n) ? sep_ids[k] : -1;
-  uint8_t* blob = static_cast<uint8_t*>(index);
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(blob, 0, sizeof(sepllm_index_header), stream));
-  dim3 grid(n_chunks, desc->B);
-  // index_count writes every chunk sum that index_scan reads, so nothing left in the array by an
-  // earlier call is ever used and nothing has to be cleared.
-  index_count<<<grid, kIdxThreads, 0, stream>>>(token_ids, desc->L, desc->n_init, sep, chunk_sums,
-                                                n_chunks);
-  index_scan<<<grid, kIdxThreads, 0, stream>>>(
-      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, chunk_sums, n_chunks,
-      desc->side_cap, reinterpret_cast<int32_t*>(blob + h.off_cnt),
-      reinterpret_cast<int32_t*>(blob + h.off_lim),
-      reinterpret_cast<int32_t*>(blob + h.off_side_pos),
-      reinterpret_cast<int32_t*>(blob + h.off_n_side), reinterpret_cast<int32_t*>(blob));
-  const int units = desc->B * h.n_tiles;
-  const int blocks = max(1, min(148 * 4, (units + 7) / 8));
-  index_tiles<<<blocks, 256, 0, stream>>>(h, blob);
-  SEPLLM_CUDA_TRY(cudaGetLastError());
-  return SEPLLM_OK;
+  if (index_scratch_words(desc->B, n_chunks) > size_t(kStaticWords)) return SEPLLM_BUFFER_TOO_SMALL;
+  int32_t* scratch = nullptr;
+  if ((st = static_chunk_sums(&scratch)) != SEPLLM_OK) return st;
+  // launch_index clears the words this call uses before the scan reads them, so nothing an
+  // earlier call left in the array matters.
+  return launch_index(desc, h, token_ids, sep_ids, static_cast<uint8_t*>(index), scratch,
+                      static_cast<cudaStream_t>(stream_));
 }

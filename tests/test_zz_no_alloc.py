@@ -29,7 +29,7 @@ def _both(ids, a, n, side_cap):
 
 
 def test_static_scratch_index_equals_regular_index_twice_in_a_row():
-    # first call: many chunks with many separators, so the shared array is left full of large sums
+    # first call: many chunks with many separators, so the shared array is left full of records
     ids1 = inputs.token_ids(21, 6, 50_000, 0.4, "iid")
     got, ref = _both(ids1, 4, 300, 50_000)
     assert torch.equal(got, ref)
@@ -43,7 +43,8 @@ def test_static_scratch_index_equals_regular_index_twice_in_a_row():
 
 
 def test_static_scratch_rejects_sizes_beyond_its_limit():
-    # 32 sequences of 2^24 ids = 131072 chunks > 65536: refused on the host, nothing launched
+    # 32 sequences of 2^24 ids need 32 * (2 * 4096 + 1) words > 65536: refused on the host,
+    # nothing launched
     desc = api.IndexDesc(32, 1 << 24, 4, 256, len(inputs.SEP_IDS), 128, 128, 1024)
     dummy = api.alloc_bytes(256)
     with pytest.raises(api.SepllmError) as e:

@@ -86,28 +86,27 @@ constexpr int kFar = 0x3fffffff;                // "never" / "unbounded" for col
 // ---------------------------------------------------------------------------
 // dQ: query-tile stationary
 // ---------------------------------------------------------------------------
-// One CTA owns one query tile of one head.  Shared-memory bandwidth is what bounds these MMAs, so
-// the stationary operands Q and dO are kept in tensor memory (packed bf16, written once by the
-// arithmetic threads straight from global memory) and only the streamed K_h / V_h half-tiles of
-// 64 keys pass through shared memory:
-//   warp 0      TMA producer: [K_h | V_h] stages of a ring
-//   warp 1      MMA issuer:   S = Q K_h^T and dP = dO V_h^T into one of two buffers (A from tensor
-//               memory), later dQ += dS K_h with dS read from the buffer it was computed in
-//   warps 4-7   dS = P (dP - Delta) of even half-tiles (thread = query row), packed bf16 over S
-//   warps 8-11  the same for odd half-tiles
+// One CTA owns one query tile of one head.  Shared-memory bandwidth and the near-empty MMA queue
+// are what bound these kernels, so the stationary operands Q and dO are kept in tensor memory
+// (packed bf16, written once by the arithmetic threads straight from global memory), only the
+// streamed K / V tiles pass through shared memory, and every MMA is 128 wide:
+//   warp 0      TMA producer: [K | V] tiles of 128 keys through a ring
+//   warp 1      MMA issuer:   S = Q K^T, dP = dO V^T (A from tensor memory), dQ += dS K
+//   warps 4-11  dS = P (dP - Delta): thread = query row, warpgroup u takes key columns
+//               [64u, 64u+64).  S is released as soon as it has been loaded so that the next
+//               tile's S MMAs run under this tile's arithmetic; dS goes over the dP columns.
 template <int D>
 struct DqCfg {
   static constexpr int NB = D / 64;
-  static constexpr int NST = 5;
-  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;   // one 64-key half-tile of K or V
-  static constexpr uint32_t kStage = 2 * kHalf;
+  static constexpr int NST = 3;
+  static constexpr uint32_t kTile = NB * kTileBlockBytes;   // one 128-key tile of K or V
+  static constexpr uint32_t kStage = 2 * kTile;
   static constexpr uint32_t kKV = 0;
   static constexpr uint32_t kBar = kKV + NST * kStage;
   static constexpr uint32_t kTotal = kBar + 512;
   static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
   // tensor-memory columns
-  static constexpr uint32_t kQt = 0, kdOt = 64, kBuf = 128, kBufStride = 128, kS = 0, kdP = 64,
-                            kdQ = 384;
+  static constexpr uint32_t kQt = 0, kdOt = 64, kS = 128, kdP = 256, kdQ = 384;
 };
 
 template <int D>
@@ -123,10 +122,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
                                              ~uintptr_t(1023));
   uint8_t* sKV = smem + C::kKV;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
-  uint64_t* bar_qdo = bars;            //       Q and dO written to tensor memory (256 threads)
+  uint64_t* bar_qdo = bars;            //       Q and dO written to tensor memory (8 warps)
   uint64_t* bar_acc = bars + 1;        //       every MMA complete
-  uint64_t* bar_sp = bars + 2;         // [2]   S and dP of buffer u complete
-  uint64_t* bar_ds = bars + 4;         // [2]   dS of buffer u written by its 128 threads
+  uint64_t* bar_sp = bars + 2;         //       S and dP of a tile complete
+  uint64_t* bar_sl = bars + 3;         //       S of a tile loaded into registers (8 warps)
+  uint64_t* bar_ds = bars + 4;         //       dS of a tile written (8 warps)
   uint64_t* bar_f = bars + 6;          // [NST] stage full
   uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 2 * NST);
@@ -140,17 +140,16 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   const int kv_plane = b * p.Hkv + hq / G;
   const int q_plane = b * p.Hq + hq;
   const int ns = g.ns, wlo = g.wlo;
-  const int n_steps = 2 * (ns + (g.whi - wlo));  // key half-tiles
-  // first key row of half-tile s in its tensor (side buffer or K/V)
-  auto half_y = [&](int s) -> int {
-    const int j = s >> 1;
-    return ((j < ns) ? j * kBN : (wlo + (j - ns)) * kBN) + (s & 1) * 64;
-  };
+  const int n_tiles = ns + (g.whi - wlo);
+  // first key row of tile j in its tensor (side buffer or K/V)
+  auto tile_y = [&](int j) -> int { return (j < ns) ? j * kBN : (wlo + (j - ns)) * kBN; };
 
   if (tid == 0) {
     mbar_init(bar_qdo, 8);
     mbar_init(bar_acc, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_ds + i, 4); }
+    mbar_init(bar_sp, 1);
+    mbar_init(bar_sl, 8);
+    mbar_init(bar_ds, 8);
     for (int i = 0; i < NST; ++i) { mbar_init(bar_f + i, 1); mbar_init(bar_e + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
@@ -177,58 +176,65 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
-      for (int s = 0; s < n_steps; ++s) {
-        const bool side = (s >> 1) < ns;
-        const int y = half_y(s);
-        const int st = s % NST;
-        if (s >= NST) wait(bar_e + st, (s / NST - 1) & 1);
+      for (int j = 0; j < n_tiles; ++j) {
+        const bool side = j < ns;
+        const int y = tile_y(j);
+        const int st = j % NST;
+        if (j >= NST) wait(bar_e + st, (j / NST - 1) & 1);
         mbar_expect_tx(bar_f + st, C::kStage);
         uint8_t* dst = sKV + st * C::kStage;
         for (int nb = 0; nb < NB; ++nb) {
-          tma_load_3d(dst + nb * kHalfBlockBytes, side ? &mapKs : &mapK, bar_f + st, nb * 64, y,
+          tma_load_3d(dst + nb * kTileBlockBytes, side ? &mapKs : &mapK, bar_f + st, nb * 64, y,
                       kv_plane);
-          tma_load_3d(dst + C::kHalf + nb * kHalfBlockBytes, side ? &mapVs : &mapV, bar_f + st,
+          tma_load_3d(dst + C::kTile + nb * kTileBlockBytes, side ? &mapVs : &mapV, bar_f + st,
                       nb * 64, y, kv_plane);
         }
       }
     } else if (warp == 1 && lane == 0) {
       // ---------------- MMA issuer ----------------
-      constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);                // K_h as K-major B of S
-      const uint32_t kt_lo0 = desc_lo(smem_u32(sKV), kHalfBlockBytes);  // K_h as MN-major B of dQ
-      auto issue_sp = [&](int s) {
-        const int st = s % NST, u = s & 1;
-        wait(bar_f + st, (s / NST) & 1);
-        tc_fence_after();
-        const uint32_t k_lo = k_lo0 + st * (C::kStage >> 4), v_lo = k_lo + (C::kHalf >> 4);
-        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
+      const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);                // K as the K-major B of S
+      const uint32_t kt_lo0 = desc_lo(smem_u32(sKV), kTileBlockBytes);  // K as the MN-major B of dQ
+      auto issue_s = [&](int j) {
+        const uint32_t k_lo = k_lo0 + (j % NST) * (C::kStage >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          umma_ts_lo(tb + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kHalfBlockBytes),
+          umma_ts_lo(tmem + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
+      };
+      auto issue_dp = [&](int j) {
+        const uint32_t v_lo = k_lo0 + (j % NST) * (C::kStage >> 4) + (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          umma_ts_lo(tb + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kHalfBlockBytes),
+          umma_ts_lo(tmem + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
-        tc_commit(bar_sp + u);
+        tc_commit(bar_sp);
       };
       wait(bar_qdo, 0);
+      wait(bar_f, 0);
       tc_fence_after();
-      if (n_steps > 0) issue_sp(0);
-      if (n_steps > 1) issue_sp(1);
-      for (int s = 0; s < n_steps; ++s) {
-        const int st = s % NST, u = s & 1;
-        wait(bar_ds + u, (s >> 1) & 1);
+      issue_s(0);
+      issue_dp(0);
+      for (int j = 0; j < n_tiles; ++j) {
+        const int st = j % NST;
+        if (j + 1 < n_tiles) {
+          // S of the next tile as soon as this tile's S has been read out
+          wait(bar_f + (j + 1) % NST, ((j + 1) / NST) & 1);
+          wait(bar_sl, j & 1);
+          tc_fence_after();
+          issue_s(j + 1);
+        }
+        wait(bar_ds, j & 1);
         tc_fence_after();
+        // dS of keys [64u, 64u+64) sits in columns 64u .. 64u+31 of the dP range
         const uint32_t kt_lo = kt_lo0 + st * (C::kStage >> 4);
-        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
-        umma_ts_lo(tmem + C::kdQ, tb + C::kS, kt_lo, idesc_dq, s > 0);
 #pragma unroll
-        for (int k = 1; k < 4; ++k)
-          umma_ts_lo(tmem + C::kdQ, tb + C::kS + k * 8, kt_lo + mnmajor_step(k), idesc_dq, 1);
+        for (int k = 0; k < kBN / 16; ++k)
+          umma_ts_lo(tmem + C::kdQ, tmem + C::kdP + (k >> 2) * 64 + (k & 3) * 8,
+                     kt_lo + mnmajor_step(k), idesc_dq, (j > 0 || k > 0));
         tc_commit(bar_e + st);
-        if (s + 2 < n_steps) issue_sp(s + 2);
+        if (j + 1 < n_tiles) issue_dp(j + 1);
       }
       tc_commit(bar_acc);
     }
@@ -258,33 +264,38 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tc_fence_before();
       mbar_arrive_warp(bar_qdo);
     }
-    // ---------------- dS of half-tiles s = u, u+2, ... ----------------
-    const uint32_t tb = tmem + lane_base + C::kBuf + u * C::kBufStride;
+    // ---------------- dS: warpgroup u takes key columns [64u, 64u+64) of every tile -----------
+    const uint32_t tS = tmem + lane_base + C::kS + u * 64;
+    const uint32_t tdP = tmem + lane_base + C::kdP + u * 64;
     const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
     const float2 stt = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
     const float neg_lse2 = -stt.x, delta_i = stt.y;
-    for (int s = u; s < n_steps; s += 2) {
-      const int j = s >> 1;
+    for (int j = 0; j < n_tiles; ++j) {
       const bool side = j < ns;
-      int c_lo = 0, c_hi = 64;
+      int c_lo = 0, c_hi = kBN;
       bool need_mask;
       if (side) {
-        c_hi = lim_i - half_y(s);
+        c_hi = lim_i - j * kBN;
         need_mask = (j >= g.side_full);
       } else {
-        const int key0 = half_y(s);
+        const int key0 = tile_y(j);
         c_hi = row - key0 + 1;
         c_lo = row - p.n_neighbor + 1 - key0;
-        need_mask = (key0 + 63 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
+        need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
       }
-      wait(bar_sp + u, (s >> 1) & 1);
+      wait(bar_sp, j & 1);
       tc_fence_after();
+      uint32_t sv[2][32];
+      tmem_ld32(tS, sv[0]);
+      tmem_ld32(tS + 32, sv[1]);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive_warp(bar_sl);  // the S columns may be overwritten from here on
       uint32_t pk[32];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        uint32_t sv[32], dp[32];
-        tmem_ld32(tb + C::kS + c * 32, sv);
-        tmem_ld32(tb + C::kdP + c * 32, dp);
+        uint32_t dp[32];
+        tmem_ld32(tdP + c * 32, dp);
         tmem_ld_wait();
         if (need_mask) {
 #pragma unroll
@@ -292,8 +303,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
             float ds[2];
 #pragma unroll
             for (int w = 0; w < 2; ++w) {
-              const int col = c * 32 + e + w;
-              float pr = ex2(fmaf(__uint_as_float(sv[e + w]), p.scale_log2, neg_lse2));
+              const int col = u * 64 + c * 32 + e + w;
+              float pr = ex2(fmaf(__uint_as_float(sv[c][e + w]), p.scale_log2, neg_lse2));
               pr = (col >= c_lo && col < c_hi) ? pr : 0.f;
               ds[w] = pr * (__uint_as_float(dp[e + w]) - delta_i);
             }
@@ -302,17 +313,18 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         } else {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, neg_lse2));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, neg_lse2));
+            const float p0 = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, neg_lse2));
             pk[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - delta_i),
                                               p1 * (__uint_as_float(dp[e + 1]) - delta_i));
           }
         }
       }
-      tmem_st32(tb + C::kS, pk);
+      // packed dS over the first half of this thread's own dP columns
+      tmem_st32(tdP, pk);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive_warp(bar_ds + u);
+      mbar_arrive_warp(bar_ds);
     }
     // ---------------- epilogue: each warpgroup stores half of the row ----------------
     wait(bar_acc, 0);
@@ -746,7 +758,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        int(DkvCfg<D>::kRequest)));
   bwd_dq_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
-      mk_h, mv_h, mks_h, mvs_h, static_cast<const __nv_bfloat16*>(Q),
+      mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q),
       static_cast<const __nv_bfloat16*>(dO), p);
   record_event(d, 3, stream);
   bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv * lay.split, d->B), kBwdThreads,

@@ -197,6 +197,36 @@ def attn_rows_fwd_bwd(Q, K, V, dO, f, a: int, n: int, rows, scale: float | None 
     return O, LSE, dQ
 
 
+def attn_keys_bwd(Q, K, V, dO, f, a: int, n: int, keys, scale: float | None = None):
+    """dK and dV of selected key positions for one query head (the caller sums
+    over the query heads that share the KV head).  Q, dO, K, V: [L][d].
+
+    A key's gradient gathers every query row that keeps it, so the rows that
+    keep at least one selected key are evaluated in full (same formulas as
+    attn_bwd_head) and only the selected columns are summed.  Used where L is
+    too long to evaluate every row; pick keys that few rows keep."""
+    keys = np.asarray(keys)
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    L, d = Q.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    first = int(keys.min())
+    cand = np.arange(first, L)
+    Mc = mask_rows(f, a, n, cand)
+    rows = cand[Mc[:, keys].any(axis=1)]
+    M = mask_rows(f, a, n, rows)
+    O, _, A = attn_fwd_rows(Q[rows], K, V, M, scale)
+    dA = dO[rows] @ V.T
+    delta = (dO[rows] * O).sum(axis=1, keepdims=True)
+    dLam = A * (dA - delta)
+    dK = (dLam[:, keys].T @ Q[rows]) * scale
+    dV = A[:, keys].T @ dO[rows]
+    return dK, dV
+
+
 # ----------------------------------------------------------------------------
 # Index (the data the kernels consume; integers, compared bit for bit)
 # ----------------------------------------------------------------------------

@@ -292,3 +292,19 @@ def test_index_invariants(L, a, n, BM, BN):
             assert (sl - 1) * BN < max(lim[i] for i in rows) <= sl * BN or (sl == 0 and max(lim[i] for i in rows) == 0)
             assert wl == max(0, rows[0] - n + 1) and wh == rows[-1] + 1
             assert tl * BN <= wl < (tl + 1) * BN and (th - 1) * BN < wh <= th * BN and z == 0
+
+
+def test_selected_key_gradients_equal_the_all_rows_backward():
+    """attn_keys_bwd (used at sizes where not every row can be evaluated) against attn_bwd_head,
+    which is pinned above by autograd and finite differences."""
+    rng = np.random.default_rng(5)
+    L, d, a, n = 90, 8, 2, 7
+    f = rng.random(L) < 0.2
+    Q, K, V, dO = (rng.standard_normal((L, d)) for _ in range(4))
+    M = orc.mask_matrix(f, a, n)
+    _, dK, dV = orc.attn_bwd_head(Q, K, V, dO, M)
+    keys = np.array([40, 41, 55, 70, 88, 89])
+    keys = np.concatenate([keys, np.flatnonzero(f)[-2:]])
+    gk, gv = orc.attn_keys_bwd(Q, K, V, dO, f, a, n, keys)
+    assert np.allclose(gk, dK[keys], rtol=1e-12, atol=1e-12)
+    assert np.allclose(gv, dV[keys], rtol=1e-12, atol=1e-12)

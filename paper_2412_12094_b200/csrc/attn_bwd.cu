@@ -80,7 +80,6 @@ __device__ __forceinline__ void store_row_chunk32(void* base, size_t elem_off, i
 }
 
 constexpr int kBwdThreads = 384;
-constexpr uint32_t kHalfBlockBytes = 64 * 128;  // 64 rows x 64 bf16, one swizzled block
 constexpr int kFar = 0x3fffffff;                // "never" / "unbounded" for column ranges
 
 // ---------------------------------------------------------------------------
@@ -124,9 +123,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
   uint64_t* bar_qdo = bars;            //       Q and dO written to tensor memory (8 warps)
   uint64_t* bar_acc = bars + 1;        //       every MMA complete
-  uint64_t* bar_sp = bars + 2;         //       S and dP of a tile complete
+  uint64_t* bar_s = bars + 2;          //       S of a tile complete
   uint64_t* bar_sl = bars + 3;         //       S of a tile loaded into registers (8 warps)
   uint64_t* bar_ds = bars + 4;         //       dS of a tile written (8 warps)
+  uint64_t* bar_dp = bars + 5;         //       dP of a tile complete
   uint64_t* bar_f = bars + 6;          // [NST] stage full
   uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 2 * NST);
@@ -147,7 +147,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   if (tid == 0) {
     mbar_init(bar_qdo, 8);
     mbar_init(bar_acc, 1);
-    mbar_init(bar_sp, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_dp, 1);
     mbar_init(bar_sl, 8);
     mbar_init(bar_ds, 8);
     for (int i = 0; i < NST; ++i) { mbar_init(bar_f + i, 1); mbar_init(bar_e + i, 1); }
@@ -202,6 +203,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
+        tc_commit(bar_s);
       };
       auto issue_dp = [&](int j) {
         const uint32_t v_lo = k_lo0 + (j % NST) * (C::kStage >> 4) + (C::kTile >> 4);
@@ -209,7 +211,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
-        tc_commit(bar_sp);
+        tc_commit(bar_dp);
       };
       wait(bar_qdo, 0);
       wait(bar_f, 0);
@@ -283,7 +285,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         c_lo = row - p.n_neighbor + 1 - key0;
         need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
       }
-      wait(bar_sp, j & 1);
+      // phase A (needs S only; runs under the previous tile's dQ and this tile's dP MMAs):
+      // P = exp2(S * scale - LSE), kept in registers
+      wait(bar_s, j & 1);
       tc_fence_after();
       uint32_t sv[2][32];
       tmem_ld32(tS, sv[0]);
@@ -291,34 +295,36 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive_warp(bar_sl);  // the S columns may be overwritten from here on
+      if (need_mask) {
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int col = u * 64 + c * 32 + e;
+            const float pr = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
+            sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? pr : 0.f);
+          }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2)));
+      }
+      // phase B: dS = P (dP - Delta)
+      wait(bar_dp, j & 1);
+      tc_fence_after();
       uint32_t pk[32];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t dp[32];
         tmem_ld32(tdP + c * 32, dp);
         tmem_ld_wait();
-        if (need_mask) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float ds[2];
-#pragma unroll
-            for (int w = 0; w < 2; ++w) {
-              const int col = u * 64 + c * 32 + e + w;
-              float pr = ex2(fmaf(__uint_as_float(sv[c][e + w]), p.scale_log2, neg_lse2));
-              pr = (col >= c_lo && col < c_hi) ? pr : 0.f;
-              ds[w] = pr * (__uint_as_float(dp[e + w]) - delta_i);
-            }
-            pk[c * 16 + (e >> 1)] = pack_bf16(ds[0], ds[1]);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, neg_lse2));
-            pk[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - delta_i),
-                                              p1 * (__uint_as_float(dp[e + 1]) - delta_i));
-          }
-        }
+        for (int e = 0; e < 32; e += 2)
+          pk[c * 16 + (e >> 1)] =
+              pack_bf16(__uint_as_float(sv[c][e]) * (__uint_as_float(dp[e]) - delta_i),
+                        __uint_as_float(sv[c][e + 1]) * (__uint_as_float(dp[e + 1]) - delta_i));
       }
       // packed dS over the first half of this thread's own dP columns
       tmem_st32(tdP, pk);
@@ -352,30 +358,34 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
 // ---------------------------------------------------------------------------
 // dK, dV: key-tile stationary
 // ---------------------------------------------------------------------------
-// One CTA owns 128 keys and streams the query rows that keep any of them, 64 rows of one query
-// head at a time ("half-iteration"), through a ring of NSTQ stages:
-//   warp 0      TMA producer (K, V once; then Q_h, dO_h per half-iteration)
-//   warp 1      MMA issuer:  S^T = K Q_h^T and dP^T = V dO_h^T into one of two tensor-memory
-//               buffers; later dV += P^T dO_h and dK += dS^T Q_h with A taken from tensor memory
-//   warps 2-3   load the 64 (LSE, Delta) pairs of the half-iteration into shared memory
-//   warps 4-7   P^T, dS^T of even half-iterations (thread = key row), written as packed bf16
-//               over the S^T / dP^T columns they came from
-//   warps 8-11  the same for odd half-iterations
+// One CTA owns 128 keys and streams the query tiles (128 rows of one query head per iteration)
+// that keep any of them:
+//   warp 0      TMA producer (K, V once; then Q and dO per iteration through rings of their own)
+//   warp 1      MMA issuer:  S^T = K Q^T, dP^T = V dO^T (128 wide), then dV += P^T dO and
+//               dK += dS^T Q with A taken from tensor memory
+//   warps 2-3   load the 128 (LSE, Delta) pairs of the iteration into shared memory
+//   warps 4-11  P^T and dS^T (thread = key row); warpgroup u takes query columns [64u, 64u+64).
+//               S^T is released as soon as it has been loaded, so the next iteration's S^T MMAs
+//               run under this iteration's arithmetic; P^T and dS^T go, packed, over the two
+//               halves of the thread's own dP^T columns.
 template <int D>
 struct DkvCfg {
   static constexpr int NB = D / 64;
-  static constexpr int NSTQ = 4;
+  // Q is needed one iteration earlier than dO (S^T runs under the previous iteration's
+  // arithmetic), so it gets the deeper ring; a tile takes about a microsecond to arrive.
+  static constexpr int NSQ = 3, NSO = 2;
   static constexpr uint32_t kTile = NB * kTileBlockBytes;
-  static constexpr uint32_t kHalf = NB * kHalfBlockBytes;
   static constexpr uint32_t kK = 0;
   static constexpr uint32_t kV = kK + kTile;
-  static constexpr uint32_t kQ = kV + kTile;                 // NSTQ x [Q_h | dO_h]
-  static constexpr uint32_t kStat = kQ + NSTQ * 2 * kHalf;   // NSTQ x 64 float2
-  static constexpr uint32_t kBar = kStat + NSTQ * 64 * 8;
+  static constexpr uint32_t kQ = kV + kTile;                 // NSQ x Q
+  static constexpr uint32_t kdO = kQ + NSQ * kTile;          // NSO x dO
+  static constexpr uint32_t kStat = kdO + NSO * kTile;       // 128 float2, one iteration at a time
+  static constexpr uint32_t kBar = kStat + 128 * 8;
   static constexpr uint32_t kTotal = kBar + 512;
   static constexpr uint32_t kRequest = (kTotal + 1024 > 116 * 1024) ? kTotal + 1024 : 116 * 1024;
+  static_assert(kRequest <= 227 * 1024, "shared memory budget");
   // tensor-memory columns
-  static constexpr uint32_t kdV = 0, kdK = D, kBuf = 256, kBufStride = 128, kST = 0, kdPT = 64;
+  static constexpr uint32_t kdV = 0, kdK = D, kST = 256, kdPT = 384;
 };
 
 template <int D, bool SIDE>
@@ -384,23 +394,28 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const BwdParams p) {
   using C = DkvCfg<D>;
-  constexpr int NB = C::NB, NSTQ = C::NSTQ;
+  constexpr int NB = C::NB, NSQ = C::NSQ, NSO = C::NSO;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
   uint8_t* sK = smem + C::kK;
   uint8_t* sV = smem + C::kV;
   uint8_t* sQ = smem + C::kQ;
+  uint8_t* sdO = smem + C::kdO;
   float2* s_stat = reinterpret_cast<float2*>(smem + C::kStat);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
   uint64_t* bar_kv = bars;              //        K, V landed
   uint64_t* bar_acc = bars + 1;         //        every MMA complete
-  uint64_t* bar_sp = bars + 2;          // [2]    S^T and dP^T of buffer u complete
-  uint64_t* bar_pds = bars + 4;         // [2]    P^T and dS^T of buffer u written
-  uint64_t* bar_qf = bars + 6;          // [NSTQ] Q_h, dO_h landed
-  uint64_t* bar_qe = bar_qf + NSTQ;     // [NSTQ] stage free (its dV / dK MMAs are complete)
-  uint64_t* bar_sf = bar_qe + NSTQ;     // [NSTQ] row statistics written
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 3 * NSTQ);
+  uint64_t* bar_st = bars + 2;          //        S^T of an iteration complete
+  uint64_t* bar_sl = bars + 3;          //        S^T loaded into registers (8 warps)
+  uint64_t* bar_pds = bars + 4;         //        P^T and dS^T written (8 warps)
+  uint64_t* bar_sf = bars + 5;          //        row statistics of an iteration written (2 warps)
+  uint64_t* bar_dpt = bars + 6;         //        dP^T of an iteration complete
+  uint64_t* bar_qf = bars + 7;          // [NSQ]  Q landed
+  uint64_t* bar_qe = bar_qf + NSQ;      // [NSQ]  Q stage free (its dK MMAs are complete)
+  uint64_t* bar_of = bar_qe + NSQ;      // [NSO]  dO landed
+  uint64_t* bar_oe = bar_of + NSO;      // [NSO]  dO stage free (its dV MMAs are complete)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 2 * NSQ + 2 * NSO);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -413,25 +428,29 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int g_lo = (split > 1) ? part : 0, n_g = (split > 1) ? 1 : G;
   const int kv_plane = b * p.Hkv + hk;
   const int ns = min(p.n_side[b], p.side_cap);
-  const int QH = (p.L + 63) / 64;
 
-  // query half-tiles [qh_lo, qh_hi] that keep at least one key of this tile
-  int qh_lo, qh_hi;
+  // query tiles [t_lo, t_hi] that keep at least one key of this tile
+  int t_lo, t_hi;
   if (SIDE) {
     if (kt * kBN >= ns) return;  // no entries in this side tile: nothing reads its partial rows
-    qh_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / 64;
-    qh_hi = QH - 1;
+    t_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / kBM;
+    t_hi = p.T - 1;
   } else {
-    qh_lo = 2 * kt;  // kBM == kBN
-    qh_hi = min(QH - 1, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / 64);
+    t_lo = kt;  // kBM == kBN
+    t_hi = min(p.T - 1, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / kBM);
   }
-  const int n_it = max(0, qh_hi - qh_lo + 1) * n_g;
+  const int n_it = max(0, t_hi - t_lo + 1) * n_g;
 
   if (tid == 0) {
     mbar_init(bar_kv, 1);
     mbar_init(bar_acc, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_sp + i, 1); mbar_init(bar_pds + i, 4); }
-    for (int i = 0; i < NSTQ; ++i) { mbar_init(bar_qf + i, 1); mbar_init(bar_qe + i, 1); mbar_init(bar_sf + i, 2); }
+    mbar_init(bar_st, 1);
+    mbar_init(bar_dpt, 1);
+    mbar_init(bar_sl, 8);
+    mbar_init(bar_pds, 8);
+    mbar_init(bar_sf, 2);
+    for (int i = 0; i < NSQ; ++i) { mbar_init(bar_qf + i, 1); mbar_init(bar_qe + i, 1); }
+    for (int i = 0; i < NSO; ++i) { mbar_init(bar_of + i, 1); mbar_init(bar_oe + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -453,7 +472,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
   };
   auto q_plane_of = [&](int it) { return b * p.Hq + hk * G + g_lo + it % n_g; };
-  auto q0_of = [&](int it) { return (qh_lo + it / n_g) * 64; };
+  auto q0_of = [&](int it) { return (t_lo + it / n_g) * kBM; };
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
@@ -465,71 +484,87 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tma_load_3d(sV + nb * kTileBlockBytes, &mapV, bar_kv, nb * 64, kt * kBN, kv_plane);
       }
       for (int it = 0; it < n_it; ++it) {
-        const int st = it % NSTQ;
-        if (it >= NSTQ) wait(bar_qe + st, (it / NSTQ - 1) & 1);
-        mbar_expect_tx(bar_qf + st, 2 * C::kHalf);
-        uint8_t* dq = sQ + st * 2 * C::kHalf;
+        const int sq = it % NSQ, so = it % NSO;
         const int y = q0_of(it), plane = q_plane_of(it);
-        for (int nb = 0; nb < NB; ++nb) {
-          tma_load_3d(dq + nb * kHalfBlockBytes, &mapQ, bar_qf + st, nb * 64, y, plane);
-          tma_load_3d(dq + C::kHalf + nb * kHalfBlockBytes, &mapdO, bar_qf + st, nb * 64, y, plane);
-        }
+        if (it >= NSQ) wait(bar_qe + sq, (it / NSQ - 1) & 1);
+        mbar_expect_tx(bar_qf + sq, C::kTile);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sQ + sq * C::kTile + nb * kTileBlockBytes, &mapQ, bar_qf + sq, nb * 64, y, plane);
+        if (it >= NSO) wait(bar_oe + so, (it / NSO - 1) & 1);
+        mbar_expect_tx(bar_of + so, C::kTile);
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_3d(sdO + so * C::kTile + nb * kTileBlockBytes, &mapdO, bar_of + so, nb * 64, y, plane);
       }
     } else if (warp == 1 && lane == 0 && n_it > 0) {
       // ---------------- MMA issuer ----------------
-      constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);
       const uint32_t k_lo = desc_lo(smem_u32(sK), 16), v_lo = desc_lo(smem_u32(sV), 16);
-      const uint32_t q_lo0 = desc_lo(smem_u32(sQ), 16);                   // Q_h, dO_h as K-major B
-      const uint32_t qt_lo0 = desc_lo(smem_u32(sQ), kHalfBlockBytes);     // ... as MN-major B
-      auto issue_sp = [&](int it) {
-        const int st = it % NSTQ, u = it & 1;
-        wait(bar_qf + st, (it / NSTQ) & 1);
+      const uint32_t q_lo0 = desc_lo(smem_u32(sQ), 16), do_lo0 = desc_lo(smem_u32(sdO), 16);  // K-major B
+      const uint32_t qt_lo0 = desc_lo(smem_u32(sQ), kTileBlockBytes);                         // MN-major B
+      const uint32_t dot_lo0 = desc_lo(smem_u32(sdO), kTileBlockBytes);
+      auto issue_st = [&](int it) {
+        const uint32_t q_lo = q_lo0 + (it % NSQ) * (C::kTile >> 4);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          umma_ss_lo(tmem + C::kST, k_lo + kmajor_step(k, kTileBlockBytes),
+                     q_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
+        tc_commit(bar_st);
+      };
+      auto issue_dpt = [&](int it) {
+        wait(bar_of + it % NSO, (it / NSO) & 1);
         tc_fence_after();
-        const uint32_t q_lo = q_lo0 + st * (2 * C::kHalf >> 4), do_lo = q_lo + (C::kHalf >> 4);
-        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
+        const uint32_t do_lo = do_lo0 + (it % NSO) * (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          umma_ss_lo(tb + C::kST, k_lo + kmajor_step(k, kTileBlockBytes),
-                     q_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          umma_ss_lo(tb + C::kdPT, v_lo + kmajor_step(k, kTileBlockBytes),
-                     do_lo + kmajor_step(k, kHalfBlockBytes), idesc_s, k > 0);
-        tc_commit(bar_sp + u);
+          umma_ss_lo(tmem + C::kdPT, v_lo + kmajor_step(k, kTileBlockBytes),
+                     do_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
+        tc_commit(bar_dpt);
       };
       wait(bar_kv, 0);
-      issue_sp(0);
-      if (n_it > 1) issue_sp(1);
+      wait(bar_qf, 0);
+      tc_fence_after();
+      issue_st(0);
+      issue_dpt(0);
       for (int it = 0; it < n_it; ++it) {
-        const int st = it % NSTQ, u = it & 1;
-        wait(bar_pds + u, (it >> 1) & 1);
+        if (it + 1 < n_it) {
+          wait(bar_qf + (it + 1) % NSQ, ((it + 1) / NSQ) & 1);
+          wait(bar_sl, it & 1);
+          tc_fence_after();
+          issue_st(it + 1);
+        }
+        wait(bar_pds, it & 1);
         tc_fence_after();
-        const uint32_t qt_lo = qt_lo0 + st * (2 * C::kHalf >> 4), dot_lo = qt_lo + (C::kHalf >> 4);
-        const uint32_t tb = tmem + C::kBuf + u * C::kBufStride;
-        umma_ts_lo(tmem + C::kdV, tb + C::kST, dot_lo, idesc_acc, it > 0);
+        // Within the dP^T range, warpgroup u's columns [64u, 64u+64) hold P^T of its 64 queries
+        // in the first 32 and dS^T in the last 32.
+        const uint32_t dot_lo = dot_lo0 + (it % NSO) * (C::kTile >> 4);
+        const uint32_t qt_lo = qt_lo0 + (it % NSQ) * (C::kTile >> 4);
 #pragma unroll
-        for (int k = 1; k < 4; ++k)
-          umma_ts_lo(tmem + C::kdV, tb + C::kST + k * 8, dot_lo + mnmajor_step(k), idesc_acc, 1);
-        umma_ts_lo(tmem + C::kdK, tb + C::kdPT, qt_lo, idesc_acc, it > 0);
+        for (int k = 0; k < kBM / 16; ++k)
+          umma_ts_lo(tmem + C::kdV, tmem + C::kdPT + (k >> 2) * 64 + (k & 3) * 8,
+                     dot_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
+        tc_commit(bar_oe + it % NSO);
 #pragma unroll
-        for (int k = 1; k < 4; ++k)
-          umma_ts_lo(tmem + C::kdK, tb + C::kdPT + k * 8, qt_lo + mnmajor_step(k), idesc_acc, 1);
-        tc_commit(bar_qe + st);
-        if (it + 2 < n_it) issue_sp(it + 2);
+        for (int k = 0; k < kBM / 16; ++k)
+          umma_ts_lo(tmem + C::kdK, tmem + C::kdPT + (k >> 2) * 64 + 32 + (k & 3) * 8,
+                     qt_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
+        tc_commit(bar_qe + it % NSQ);
+        if (it + 1 < n_it) issue_dpt(it + 1);
       }
       tc_commit(bar_acc);
     } else if (warp >= 2) {
       // ---------------- row statistics ----------------
+      // one buffer: iteration it's pairs are written once iteration it-1's arithmetic is done
       const int i = tid - 64;  // 0..63
       for (int it = 0; it < n_it; ++it) {
-        const int st = it % NSTQ;
         const int q = q0_of(it) + i;
-        const float2 v = (q < p.L) ? p.stats[size_t(q_plane_of(it)) * p.L + q]
-                                   : make_float2(INFINITY, 0.f);
-        if (it >= NSTQ) wait(bar_qe + st, (it / NSTQ - 1) & 1);
-        s_stat[st * 64 + i] = make_float2(-v.x, v.y);
-        mbar_arrive_warp(bar_sf + st);
+        const size_t base = size_t(q_plane_of(it)) * p.L;
+        const float2 v0 = (q < p.L) ? p.stats[base + q] : make_float2(INFINITY, 0.f);
+        const float2 v1 = (q + 64 < p.L) ? p.stats[base + q + 64] : make_float2(INFINITY, 0.f);
+        if (it >= 1) wait(bar_pds, (it - 1) & 1);
+        s_stat[i] = make_float2(-v0.x, v0.y);
+        s_stat[64 + i] = make_float2(-v1.x, v1.y);
+        mbar_arrive_warp(bar_sf);
       }
     }
   } else {
@@ -539,7 +574,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const int r = tid & 127;
     const int key = kt * kBN + r;  // side entry index (SIDE) or key position (window)
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-    const uint32_t tb = tmem + lane_base + C::kBuf + u * C::kBufStride;
+    const uint32_t tST = tmem + lane_base + C::kST + u * 64;
+    const uint32_t tdPT = tmem + lane_base + C::kdPT + u * 64;
     // queries that keep this key: [q_first, q_first + span)
     int q_first, span, tile_q_max;
     if (SIDE) {
@@ -554,55 +590,70 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       span = p.n_neighbor;
       tile_q_max = 0;
     }
-    for (int it = u; it < n_it; it += 2) {
-      const int st = it % NSTQ;
+    for (int it = 0; it < n_it; ++it) {
       const int q0 = q0_of(it);
       const int c_lo = q_first - q0, c_hi = c_lo + span;
       bool need_mask;
       if (SIDE) need_mask = tile_q_max > q0;
-      else need_mask = !(kt * kBN + kBN - 1 <= q0 && q0 + 63 <= kt * kBN + p.n_neighbor - 1);
-      wait(bar_sf + st, (it / NSTQ) & 1);
-      wait(bar_sp + u, (it >> 1) & 1);
+      else need_mask = !(kt * kBN + kBN - 1 <= q0 && q0 + kBM - 1 <= kt * kBN + p.n_neighbor - 1);
+      // phase A (needs S^T only; runs under the previous iteration's dV / dK and this iteration's
+      // dP^T MMAs): P^T = exp2(S^T * scale - LSE), kept in registers
+      wait(bar_sf, it & 1);
+      wait(bar_st, it & 1);
       tc_fence_after();
+      uint32_t sv[2][32];
+      tmem_ld32(tST, sv[0]);
+      tmem_ld32(tST + 32, sv[1]);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive_warp(bar_sl);  // the S^T columns may be overwritten from here on
       // two columns' (-LSE in log2 units, Delta) per shared-memory load
-      const float4* stat2 = reinterpret_cast<const float4*>(s_stat + st * 64);
-      uint32_t pkp[32], pkd[32];
+      const float4* stat2 = reinterpret_cast<const float4*>(s_stat + u * 64);
+      if (need_mask) {
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t sv[32], dp[32];
-        tmem_ld32(tb + C::kST + c * 32, sv);
-        tmem_ld32(tb + C::kdPT + c * 32, dp);
-        tmem_ld_wait();
-        if (need_mask) {
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const int col = c * 32 + e;
-            const float4 sd = stat2[col >> 1];
-            float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, sd.x));
-            float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, sd.z));
-            p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
-            p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
-            pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
-            pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
-                                               p1 * (__uint_as_float(dp[e + 1]) - sd.w));
+            const int col = u * 64 + c * 32 + e;
+            const float4 sd = stat2[(c * 32 + e) >> 1];
+            const float p0 = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, sd.x));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, sd.z));
+            sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? p0 : 0.f);
+            sv[c][e + 1] = __float_as_uint((col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f);
           }
-        } else {
+      } else {
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             const float4 sd = stat2[(c * 32 + e) >> 1];
-            const float p0 = ex2(fmaf(__uint_as_float(sv[e]), p.scale_log2, sd.x));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, sd.z));
-            pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
-            pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
-                                               p1 * (__uint_as_float(dp[e + 1]) - sd.w));
+            sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, sd.x)));
+            sv[c][e + 1] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, sd.z)));
           }
+      }
+      // phase B: dS^T = P^T (dP^T - Delta)
+      wait(bar_dpt, it & 1);
+      tc_fence_after();
+      uint32_t pkp[32], pkd[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t dp[32];
+        tmem_ld32(tdPT + c * 32, dp);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float4 sd = stat2[(c * 32 + e) >> 1];
+          const float p0 = __uint_as_float(sv[c][e]), p1 = __uint_as_float(sv[c][e + 1]);
+          pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
+          pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
+                                             p1 * (__uint_as_float(dp[e + 1]) - sd.w));
         }
       }
-      tmem_st32(tb + C::kST, pkp);
-      tmem_st32(tb + C::kdPT, pkd);
+      tmem_st32(tdPT, pkp);
+      tmem_st32(tdPT + 32, pkd);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive_warp(bar_pds + u);
+      mbar_arrive_warp(bar_pds);
     }
 
     // ---------------- epilogue: warps 4-7 take dV, warps 8-11 take dK ----------------
@@ -704,8 +755,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   }
   record_event(d, 2, stream);
 
-  // 128-row boxes for the stationary operand of each pass, 64-row boxes for the streamed one
-  CUtensorMap mq, mdo, mk, mv, mks, mvs, mq_h, mdo_h, mk_h, mv_h, mks_h, mvs_h;
+  CUtensorMap mq, mdo, mk, mv, mks, mvs;
   sepllm_status st;
   const int64_t L = d->L, nq = int64_t(d->B) * d->Hq, nkv = int64_t(d->B) * d->Hkv;
   const int64_t cp = lay.cap_pad;
@@ -715,12 +765,6 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   if ((st = make_tile_map(&mv, V, D, L, nkv, D, L * D, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mks, Ks, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mvs, Vs, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mq_h, Q, D, L, nq, D, L * D, 64)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mdo_h, dO, D, L, nq, D, L * D, 64)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mk_h, K, D, L, nkv, D, L * D, 64)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mv_h, V, D, L, nkv, D, L * D, 64)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mks_h, Ks, D, cp, nkv, D, cp * D, 64)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mvs_h, Vs, D, cp, nkv, D, cp * D, 64)) != SEPLLM_OK) return st;
 
   BwdParams p;
   p.cnt = reinterpret_cast<const int32_t*>(index + ih.off_cnt);
@@ -762,10 +806,10 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
       static_cast<const __nv_bfloat16*>(dO), p);
   record_event(d, 3, stream);
   bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv * lay.split, d->B), kBwdThreads,
-                            DkvCfg<D>::kRequest, stream>>>(mq_h, mdo_h, mks, mvs, p);
+                            DkvCfg<D>::kRequest, stream>>>(mq, mdo, mks, mvs, p);
   record_event(d, 4, stream);
   bwd_dkv_kernel<D, false><<<dim3(ih.n_tiles, d->Hkv, d->B), kBwdThreads, DkvCfg<D>::kRequest,
-                             stream>>>(mq_h, mdo_h, mk, mv, p);
+                             stream>>>(mq, mdo, mk, mv, p);
   record_event(d, 5, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;

@@ -60,7 +60,7 @@ struct BwdParams {
   void* dK;
   void* dV;
   int32_t* status;
-  int L, T, Hq, Hkv, n_neighbor, side_cap, cap_pad, grad_fp32, split, pair_heads;
+  int B, L, T, Hq, Hkv, n_neighbor, side_cap, cap_pad, grad_fp32, split, pair_heads;
   float scale, scale_log2;
 };
 
@@ -133,9 +133,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = blockIdx.z, hq = blockIdx.y;
+  // grid (heads x batch, tiles): longest tiles first over the whole launch, and the heads of a
+  // GQA group run side by side on the same K/V tiles
+  const int b = int(blockIdx.x) / p.Hq, hq = int(blockIdx.x) % p.Hq;
   const int G = p.Hq / p.Hkv;
-  const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
+  const int t = p.T - 1 - int(blockIdx.y);  // long tiles first
   const SlotGeom g = load_slot(p.tile_meta, b, p.T, t, hq, p.cap_pad / kBN);
   const int kv_plane = b * p.Hkv + hq / G;
   const int q_plane = b * p.Hq + hq;
@@ -419,12 +421,15 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kt = SIDE ? int(blockIdx.x) : int(gridDim.x) - 1 - int(blockIdx.x);
-  const int b = blockIdx.z;
+  // grid (kv heads [x parts] x batch, key tiles): key tiles with the most query tiles first
+  // (side tile 0 is kept by every later query; the last window tile by the fewest)
+  const int kt = SIDE ? int(blockIdx.y) : int(gridDim.y) - 1 - int(blockIdx.y);
   const int G = p.Hq / p.Hkv;
   // the side pass may give each query head of the group its own CTA (and partial buffer)
   const int split = SIDE ? p.split : 1;
-  const int hk = int(blockIdx.y) / split, part = int(blockIdx.y) % split;
+  const int n_x = p.Hkv * split;
+  const int b = int(blockIdx.x) / n_x;
+  const int hk = (int(blockIdx.x) % n_x) / split, part = int(blockIdx.x) % split;
   const int g_lo = (split > 1) ? part : 0, n_g = (split > 1) ? 1 : G;
   const int kv_plane = b * p.Hkv + hk;
   const int ns = min(p.n_side[b], p.side_cap);
@@ -667,7 +672,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       // fp32 partial rows for the entries of this side tile
       const bool r_ok = key < p.cap_pad;
       float* base = (u ? p.dKs : p.dVs) +
-                    ((size_t(part) * gridDim.z + b) * p.Hkv + hk) * size_t(p.cap_pad) * D +
+                    ((size_t(part) * p.B + b) * p.Hkv + hk) * size_t(p.cap_pad) * D +
                     size_t(key) * D;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -695,7 +700,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int c0 = cnt_b[key], c1 = cnt_b[key + 1];
         if (c1 > c0 && c0 < ns) side_idx = c0;
       }
-      const size_t part_stride = size_t(gridDim.z) * p.Hkv * size_t(p.cap_pad) * D;
+      const size_t part_stride = size_t(p.B) * p.Hkv * size_t(p.cap_pad) * D;
       const float* part0 = (u ? p.dKs : p.dVs) +
                            (size_t(b) * p.Hkv + hk) * size_t(p.cap_pad) * D +
                            size_t(max(side_idx, 0)) * D;
@@ -779,6 +784,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.dK = dK;
   p.dV = dV;
   p.status = reinterpret_cast<int32_t*>(ws);
+  p.B = d->B;
   p.L = d->L;
   p.T = ih.n_tiles;
   p.Hq = d->Hq;
@@ -801,14 +807,14 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        int(DkvCfg<D>::kRequest)));
-  bwd_dq_kernel<D><<<dim3(ih.n_tiles, d->Hq, d->B), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
+  bwd_dq_kernel<D><<<dim3(d->Hq * d->B, ih.n_tiles), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
       mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q),
       static_cast<const __nv_bfloat16*>(dO), p);
   record_event(d, 3, stream);
-  bwd_dkv_kernel<D, true><<<dim3(lay.cap_pad / kBN, d->Hkv * lay.split, d->B), kBwdThreads,
+  bwd_dkv_kernel<D, true><<<dim3(d->Hkv * lay.split * d->B, lay.cap_pad / kBN), kBwdThreads,
                             DkvCfg<D>::kRequest, stream>>>(mq, mdo, mks, mvs, p);
   record_event(d, 4, stream);
-  bwd_dkv_kernel<D, false><<<dim3(ih.n_tiles, d->Hkv, d->B), kBwdThreads, DkvCfg<D>::kRequest,
+  bwd_dkv_kernel<D, false><<<dim3(d->Hkv * d->B, ih.n_tiles), kBwdThreads, DkvCfg<D>::kRequest,
                              stream>>>(mq, mdo, mk, mv, p);
   record_event(d, 5, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());

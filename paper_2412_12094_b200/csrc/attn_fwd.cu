@@ -144,19 +144,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = blockIdx.z;
+  // grid (heads x batch, tiles): consecutive CTAs take the same tile position of every head and
+  // sequence, longest tiles first, so work is handed out longest-first over the whole launch and
+  // the heads of a GQA group find their K/V tiles in L2
   const int G = p.Hq / p.Hkv;
+  const int heads_x = p.pair_heads ? p.Hq / 2 : p.Hq;
+  const int b = int(blockIdx.x) / heads_x, hx = int(blockIdx.x) % heads_x;
 
   // the two slots of this CTA (slot 1 is never empty; slot 0 is when T is odd and tiles pair up)
   SlotGeom g0, g1;
   if (p.pair_heads) {
-    const int t = p.T - 1 - int(blockIdx.x);  // long tiles first
-    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y), p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * int(blockIdx.y) + 1, p.side_tiles_cap);
+    const int t = p.T - 1 - int(blockIdx.y);
+    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * hx, p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * hx + 1, p.side_tiles_cap);
   } else {
-    const int t = p.T - 1 - 2 * int(blockIdx.x);
-    g0 = load_slot(p.tile_meta, b, p.T, t - 1, int(blockIdx.y), p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, b, p.T, t, int(blockIdx.y), p.side_tiles_cap);
+    const int t = p.T - 1 - 2 * int(blockIdx.y);
+    g0 = load_slot(p.tile_meta, b, p.T, t - 1, hx, p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, b, p.T, t, hx, p.side_tiles_cap);
   }
   const int kv_plane = b * p.Hkv + g1.hq / G;
   // key tiles of the CTA: side tiles [0, ns), then window tiles [wlo, whi)
@@ -416,7 +420,7 @@ sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id)
   if (d->d != 64 && d->d != 128) return SEPLLM_UNSUPPORTED;
   if (id->BM != kBM || id->BN != kBN) return SEPLLM_UNSUPPORTED;
   if (d->grad_dtype != 0 && d->grad_dtype != 1) return SEPLLM_INVALID_ARG;
-  if (d->Hq > 65535 || d->B > 65535) return SEPLLM_UNSUPPORTED;
+  if (d->Hq > 65535 || d->B > 65535 || (d->L + kBM - 1) / kBM > 65535) return SEPLLM_UNSUPPORTED;
   return SEPLLM_OK;
 }
 
@@ -501,8 +505,8 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   const uint32_t smem = FwdCfg<D>::kRequest;
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_kernel<D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-  const dim3 grid = p.pair_heads ? dim3(ih.n_tiles, d->Hq / 2, d->B)
-                                 : dim3((ih.n_tiles + 1) / 2, d->Hq, d->B);
+  const dim3 grid = p.pair_heads ? dim3(d->Hq / 2 * d->B, ih.n_tiles)
+                                 : dim3(d->Hq * d->B, (ih.n_tiles + 1) / 2);
   attn_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(mq, mk, mv, mks, mvs, p);
   record_event(d, 2, stream);
   SEPLLM_CUDA_TRY(cudaGetLastError());

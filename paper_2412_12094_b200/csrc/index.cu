@@ -37,6 +37,35 @@ __device__ __forceinline__ bool in_sep_list(int32_t tok, const SepIds& s) {
   return f;
 }
 
+// Separator ids as a collision-free multiplicative hash table: slot (id * mult) >> (32 - bits)
+// holds the id; empty slots hold the first id (a token equal to it hashes to its own slot, so the
+// filler never makes a false match).  One multiply, one shift, one shared-memory load and one
+// compare per token instead of one compare per separator id.
+constexpr int kSepTableBits = 9;
+constexpr int kSepTableSize = 1 << kSepTableBits;
+struct SepTable {
+  uint32_t mult;
+  int32_t slot[kSepTableSize];
+};
+
+// Fills `t` for the (non-empty) id list; false if no multiplier of the tried ones separates them.
+static bool build_sep_table(const int32_t* ids, int n, SepTable* t) {
+  for (uint32_t trial = 0; trial < 4096; ++trial) {
+    const uint32_t mult = 0x9E3779B1u * (2 * trial + 1);
+    for (int k = 0; k < kSepTableSize; ++k) t->slot[k] = ids[0];
+    bool used[kSepTableSize] = {};
+    bool ok = true;
+    for (int k = 0; k < n && ok; ++k) {
+      const uint32_t h = (uint32_t(ids[k]) * mult) >> (32 - kSepTableBits);
+      if (used[h] && t->slot[h] != ids[k]) ok = false;  // a repeated id may share its slot
+      used[h] = true;
+      t->slot[h] = ids[k];
+    }
+    if (ok) { t->mult = mult; return true; }
+  }
+  return false;
+}
+
 // Scratch words per call: one 64-bit chunk record (state << 32 | count) per chunk, then one
 // ticket counter per sequence.  Zeroed before the scan kernel runs.
 constexpr uint32_t kChunkAggregate = 1, kChunkPrefix = 2;
@@ -57,9 +86,11 @@ __device__ __forceinline__ void st_chunk_state(unsigned long long* p, uint32_t s
 constexpr int kLookbackSpins = 1 << 22;
 constexpr int kMaxTilesPerChunk = kIdxChunk / kIdxPerThread + 2;  // query tiles of >= 16 rows under one chunk
 
+// NS >= 0: compare against the first NS list entries; NS < 0: look the token up in `tab`.
 template <int NS>
 __global__ void __launch_bounds__(kIdxThreads)
 index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neighbor, SepIds sep,
+           const __grid_constant__ SepTable tab,
            unsigned long long* __restrict__ chunk_state, int32_t* __restrict__ tickets,
            int n_chunks, int side_cap, int32_t* __restrict__ cnt, int32_t* __restrict__ lim,
            int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
@@ -72,8 +103,17 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   __shared__ int32_t tile_part[kMaxTilesPerChunk];
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  __shared__ int32_t tab_s[(NS < 0) ? kSepTableSize : 1];
+  __shared__ int lb_sum[kIdxThreads / 32], lb_found[kIdxThreads / 32];
   if (tid == 0) s_chunk = atomicAdd(&tickets[b], 1);
+  if (NS < 0) {
+    for (int k = tid; k < kSepTableSize; k += kIdxThreads) tab_s[k] = tab.slot[k];
+  }
   __syncthreads();
+  auto is_sep = [&](int32_t tok) -> bool {
+    if (NS < 0) return tab_s[(uint32_t(tok) * tab.mult) >> (32 - kSepTableBits)] == tok;
+    return in_sep_list<(NS < 0 ? 0 : NS)>(tok, sep);
+  };
   const int chunk = s_chunk;
   if (chunk >= n_chunks) return;
   const int32_t* ids = token_ids + static_cast<size_t>(b) * L;
@@ -87,15 +127,15 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int4 v = src[q];
-      fl |= uint32_t(in_sep_list<NS>(v.x, sep)) << (4 * q);
-      fl |= uint32_t(in_sep_list<NS>(v.y, sep)) << (4 * q + 1);
-      fl |= uint32_t(in_sep_list<NS>(v.z, sep)) << (4 * q + 2);
-      fl |= uint32_t(in_sep_list<NS>(v.w, sep)) << (4 * q + 3);
+      fl |= uint32_t(is_sep(v.x)) << (4 * q);
+      fl |= uint32_t(is_sep(v.y)) << (4 * q + 1);
+      fl |= uint32_t(is_sep(v.z)) << (4 * q + 2);
+      fl |= uint32_t(is_sep(v.w)) << (4 * q + 3);
     }
   } else {
 #pragma unroll
     for (int k = 0; k < kIdxPerThread; ++k)
-      if (j0 + k < L) fl |= uint32_t(in_sep_list<NS>(ids[j0 + k], sep)) << k;
+      if (j0 + k < L) fl |= uint32_t(is_sep(ids[j0 + k])) << k;
   }
   if (j0 < n_init) {  // initial tokens are side members too
     const int m = max(0, min(kIdxPerThread, min(n_init, L) - j0));
@@ -119,39 +159,9 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
     total += warp_buf[k];
   }
 
-  // Chunk-relative counts go to shared memory while warp 0 looks back over the earlier chunks of
-  // the sequence for the number of side members before this chunk.
-  if (wid == 0) {
-    unsigned long long* st = chunk_state + static_cast<size_t>(b) * n_chunks;
-    int off = 0;
-    if (chunk > 0) {
-      if (lane == 0) st_chunk_state(st + chunk, kChunkAggregate, total);
-      int look = chunk - 1;
-      int spins = 0;
-      bool gave_up = false;
-      while (look >= 0) {
-        const int c = look - lane;
-        unsigned long long v = (c >= 0) ? ld_chunk_state(st + c)
-                                        : (static_cast<unsigned long long>(kChunkPrefix) << 32);
-        const uint32_t state = uint32_t(v >> 32);
-        if (__any_sync(0xffffffffu, state == 0)) {  // a predecessor has not published yet
-          if (++spins > kLookbackSpins) { gave_up = true; break; }
-          __nanosleep(64);
-          continue;
-        }
-        const uint32_t prefix_mask = __ballot_sync(0xffffffffu, state == kChunkPrefix);
-        const int first = prefix_mask ? __ffs(prefix_mask) - 1 : 32;  // nearest chunk holding a prefix
-        off += warp_sum((lane <= first) ? int(uint32_t(v)) : 0);
-        if (prefix_mask) break;
-        look -= 32;
-      }
-      if (gave_up && lane == 0) set_status(status, SEPLLM_TIMEOUT);
-    }
-    if (lane == 0) {
-      st_chunk_state(st + chunk, kChunkPrefix, off + total);
-      s_off = off;
-    }
-  }
+  // publish this chunk's count at once so that later chunks need not wait for its look-back
+  unsigned long long* st = chunk_state + static_cast<size_t>(b) * n_chunks;
+  if (tid == 0 && chunk > 0) st_chunk_state(st + chunk, kChunkAggregate, total);
   // Position p of the chunk is the lim of row base + shift + p; with BM >= 16 a thread's 16 rows
   // lie in at most two query tiles, whose side-pair sums are gathered in shared memory.
   const int shift = n_neighbor - 1;
@@ -179,6 +189,43 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
       const int tl = int((row_lo + p0) / BM) - t_first;
       if (s0) atomicAdd(&tile_part[tl], s0);
       if (s1) atomicAdd(&tile_part[tl + 1], s1);
+    }
+  }
+  // Side members before this chunk: every thread looks at one earlier chunk (warp w at chunks
+  // chunk-1-32w .. chunk-32-32w), so the whole look-back is one round trip to L2 when the records
+  // are there; a warp waits only for records not yet published.  The sum runs back to the nearest
+  // chunk that already holds a prefix.
+  {
+    int off_acc = 0;
+    bool gave_up = false;
+    for (int look = chunk - 1; look >= 0; look -= kIdxThreads) {
+      const int c = look - tid;
+      unsigned long long v = static_cast<unsigned long long>(kChunkPrefix) << 32;  // before chunk 0
+      int spins = 0;
+      while (true) {
+        if (c >= 0) v = ld_chunk_state(st + c);
+        if (!__any_sync(0xffffffffu, uint32_t(v >> 32) == 0)) break;
+        if (++spins > kLookbackSpins) { gave_up = true; break; }
+        __nanosleep(64);
+      }
+      const uint32_t prefix_mask = __ballot_sync(0xffffffffu, uint32_t(v >> 32) == kChunkPrefix);
+      const int first = prefix_mask ? __ffs(prefix_mask) - 1 : 32;
+      const int wsum = warp_sum((lane <= first) ? int(uint32_t(v)) : 0);
+      __syncthreads();  // the previous round's results have been read
+      if (lane == 0) { lb_sum[wid] = wsum; lb_found[wid] = prefix_mask != 0; }
+      __syncthreads();
+      bool done = false;
+#pragma unroll
+      for (int w = 0; w < kIdxThreads / 32; ++w) {
+        if (!done) off_acc += lb_sum[w];
+        done = done || lb_found[w];
+      }
+      if (done) break;
+    }
+    if (gave_up) set_status(status, SEPLLM_TIMEOUT);
+    if (tid == 0) {
+      st_chunk_state(st + chunk, kChunkPrefix, off_acc + total);
+      s_off = off_acc;
     }
   }
   __syncthreads();
@@ -363,14 +410,19 @@ static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_in
   dim3 grid(n_chunks, desc->B);
 #define SEPLLM_SCAN(NS)                                                                          \
   index_scan<NS><<<grid, kIdxThreads, 0, stream>>>(                                              \
-      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, chunk_state, tickets, n_chunks,   \
+      token_ids, desc->L, desc->n_init, desc->n_neighbor, sep, tab, chunk_state, tickets,        \
+      n_chunks,                                                                                  \
       desc->side_cap, reinterpret_cast<int32_t*>(blob + h.off_cnt),                              \
       reinterpret_cast<int32_t*>(blob + h.off_lim),                                              \
       reinterpret_cast<int32_t*>(blob + h.off_side_pos),                                         \
       reinterpret_cast<int32_t*>(blob + h.off_n_side),                                           \
       reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM,                   \
       reinterpret_cast<int32_t*>(blob))
+  SepTable tab;
+  tab.mult = 0;
+  const bool hashed = sep.n > 0 && build_sep_table(sep_ids, sep.n, &tab);
   if (sep.n == 0) SEPLLM_SCAN(0);
+  else if (hashed) SEPLLM_SCAN(-1);
   else if (sep.n <= 8) SEPLLM_SCAN(8);
   else if (sep.n <= 12) SEPLLM_SCAN(12);
   else if (sep.n <= 16) SEPLLM_SCAN(16);

@@ -13,6 +13,8 @@
 //                 of being the target of contended atomics.  The side pass runs first and leaves
 //                 fp32 partial rows; the window pass adds them to the rows of the same tokens
 //                 before rounding once to the output type.
+#include <algorithm>
+
 #include "attn_common.cuh"
 
 namespace sepllm {
@@ -108,12 +110,39 @@ struct DqCfg {
   static constexpr uint32_t kQt = 0, kdOt = 64, kS = 128, kdP = 256, kdQ = 384;
 };
 
+// One unit of work of the dQ kernel: a query tile of one head.
+struct DqItem {
+  int t, kv_plane, q_plane, b, ns, wlo, n_tiles, side_full;
+};
+// Items are numbered tile-major (longest tiles first), heads x batch minor, so that the heads of
+// a GQA group work on the same K/V tiles at the same time.
+__device__ __forceinline__ DqItem dq_item(const BwdParams& p, int w) {
+  const int hb = p.Hq * p.B;
+  const int x = w % hb;
+  DqItem it;
+  it.b = x / p.Hq;
+  const int hq = x % p.Hq;
+  it.t = p.T - 1 - w / hb;
+  const SlotGeom g = load_slot(p.tile_meta, it.b, p.T, it.t, hq, p.cap_pad / kBN);
+  it.kv_plane = it.b * p.Hkv + hq / (p.Hq / p.Hkv);
+  it.q_plane = it.b * p.Hq + hq;
+  it.ns = g.ns;
+  it.wlo = g.wlo;
+  it.n_tiles = g.ns + (g.whi - g.wlo);
+  it.side_full = g.side_full;
+  return it;
+}
+
+// Persistent: one CTA per SM walks items w = blockIdx.x, blockIdx.x + gridDim.x, ...  Stage and
+// barrier phases run on a tile count that continues across items; the next item's Q and dO go
+// into tensor memory as soon as the current item's last S / dP MMAs are complete, and its first
+// MMAs run while the current item's dQ is still being stored.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
               const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
               const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ dOg,
-              const BwdParams p) {
+              const BwdParams p, const int n_items) {
   using C = DqCfg<D>;
   constexpr int NB = C::NB, NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
@@ -121,30 +150,19 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
                                              ~uintptr_t(1023));
   uint8_t* sKV = smem + C::kKV;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBar);
-  uint64_t* bar_qdo = bars;            //       Q and dO written to tensor memory (8 warps)
-  uint64_t* bar_acc = bars + 1;        //       every MMA complete
+  uint64_t* bar_qdo = bars;            //       Q and dO of an item written to tensor memory (8 warps)
+  uint64_t* bar_acc = bars + 1;        //       every MMA of an item complete
   uint64_t* bar_s = bars + 2;          //       S of a tile complete
   uint64_t* bar_sl = bars + 3;         //       S of a tile loaded into registers (8 warps)
   uint64_t* bar_ds = bars + 4;         //       dS of a tile written (8 warps)
   uint64_t* bar_dp = bars + 5;         //       dP of a tile complete
-  uint64_t* bar_f = bars + 6;          // [NST] stage full
+  uint64_t* bar_dqf = bars + 6;        //       dQ of an item read out of tensor memory (8 warps)
+  uint64_t* bar_f = bars + 7;          // [NST] stage full
   uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 2 * NST);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 2 * NST);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // grid (heads x batch, tiles): longest tiles first over the whole launch, and the heads of a
-  // GQA group run side by side on the same K/V tiles
-  const int b = int(blockIdx.x) / p.Hq, hq = int(blockIdx.x) % p.Hq;
-  const int G = p.Hq / p.Hkv;
-  const int t = p.T - 1 - int(blockIdx.y);  // long tiles first
-  const SlotGeom g = load_slot(p.tile_meta, b, p.T, t, hq, p.cap_pad / kBN);
-  const int kv_plane = b * p.Hkv + hq / G;
-  const int q_plane = b * p.Hq + hq;
-  const int ns = g.ns, wlo = g.wlo;
-  const int n_tiles = ns + (g.whi - wlo);
-  // first key row of tile j in its tensor (side buffer or K/V)
-  auto tile_y = [&](int j) -> int { return (j < ns) ? j * kBN : (wlo + (j - ns)) * kBN; };
 
   if (tid == 0) {
     mbar_init(bar_qdo, 8);
@@ -153,6 +171,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     mbar_init(bar_dp, 1);
     mbar_init(bar_sl, 8);
     mbar_init(bar_ds, 8);
+    mbar_init(bar_dqf, 8);
     for (int i = 0; i < NST; ++i) { mbar_init(bar_f + i, 1); mbar_init(bar_e + i, 1); }
     *abort_flag = 0;
     fence_mbar_init();
@@ -179,19 +198,24 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     if (warp == 0 && lane == 0) {
       // ---------------- TMA producer ----------------
-      for (int j = 0; j < n_tiles; ++j) {
-        const bool side = j < ns;
-        const int y = tile_y(j);
-        const int st = j % NST;
-        if (j >= NST) wait(bar_e + st, (j / NST - 1) & 1);
-        mbar_expect_tx(bar_f + st, C::kStage);
-        uint8_t* dst = sKV + st * C::kStage;
-        for (int nb = 0; nb < NB; ++nb) {
-          tma_load_3d(dst + nb * kTileBlockBytes, side ? &mapKs : &mapK, bar_f + st, nb * 64, y,
-                      kv_plane);
-          tma_load_3d(dst + C::kTile + nb * kTileBlockBytes, side ? &mapVs : &mapV, bar_f + st,
-                      nb * 64, y, kv_plane);
+      int tb = 0;  // tiles before this item
+      for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
+        const DqItem it = dq_item(p, w);
+        for (int j = 0; j < it.n_tiles; ++j) {
+          const bool side = j < it.ns;
+          const int y = side ? j * kBN : (it.wlo + (j - it.ns)) * kBN;
+          const int gi = tb + j, st = gi % NST;
+          if (gi >= NST) wait(bar_e + st, (gi / NST - 1) & 1);
+          mbar_expect_tx(bar_f + st, C::kStage);
+          uint8_t* dst = sKV + st * C::kStage;
+          for (int nb = 0; nb < NB; ++nb) {
+            tma_load_3d(dst + nb * kTileBlockBytes, side ? &mapKs : &mapK, bar_f + st, nb * 64, y,
+                        it.kv_plane);
+            tma_load_3d(dst + C::kTile + nb * kTileBlockBytes, side ? &mapVs : &mapV, bar_f + st,
+                        nb * 64, y, it.kv_plane);
+          }
         }
+        tb += it.n_tiles;
       }
     } else if (warp == 1 && lane == 0) {
       // ---------------- MMA issuer ----------------
@@ -199,60 +223,68 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
       const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);                // K as the K-major B of S
       const uint32_t kt_lo0 = desc_lo(smem_u32(sKV), kTileBlockBytes);  // K as the MN-major B of dQ
-      auto issue_s = [&](int j) {
-        const uint32_t k_lo = k_lo0 + (j % NST) * (C::kStage >> 4);
+      auto issue_s = [&](int gi) {
+        const uint32_t k_lo = k_lo0 + (gi % NST) * (C::kStage >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
         tc_commit(bar_s);
       };
-      auto issue_dp = [&](int j) {
-        const uint32_t v_lo = k_lo0 + (j % NST) * (C::kStage >> 4) + (C::kTile >> 4);
+      auto issue_dp = [&](int gi) {
+        const uint32_t v_lo = k_lo0 + (gi % NST) * (C::kStage >> 4) + (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
         tc_commit(bar_dp);
       };
-      wait(bar_qdo, 0);
-      wait(bar_f, 0);
-      tc_fence_after();
-      issue_s(0);
-      issue_dp(0);
-      for (int j = 0; j < n_tiles; ++j) {
-        const int st = j % NST;
-        if (j + 1 < n_tiles) {
-          // S of the next tile as soon as this tile's S has been read out
-          wait(bar_f + (j + 1) % NST, ((j + 1) / NST) & 1);
-          wait(bar_sl, j & 1);
-          tc_fence_after();
-          issue_s(j + 1);
-        }
-        wait(bar_ds, j & 1);
+      int tb = 0, ino = 0;
+      for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++ino) {
+        const int n_tiles = dq_item(p, w).n_tiles;
+        wait(bar_qdo, ino & 1);
+        wait(bar_f + tb % NST, (tb / NST) & 1);
         tc_fence_after();
-        // dS of keys [64u, 64u+64) sits in columns 64u .. 64u+31 of the dP range
-        const uint32_t kt_lo = kt_lo0 + st * (C::kStage >> 4);
+        issue_s(tb);
+        issue_dp(tb);
+        for (int j = 0; j < n_tiles; ++j) {
+          const int gi = tb + j, st = gi % NST;
+          if (j + 1 < n_tiles) {
+            // S of the next tile as soon as this tile's S has been read out
+            wait(bar_f + (gi + 1) % NST, ((gi + 1) / NST) & 1);
+            wait(bar_sl, gi & 1);
+            tc_fence_after();
+            issue_s(gi + 1);
+          }
+          wait(bar_ds, gi & 1);
+          if (j == 0 && ino > 0) wait(bar_dqf, (ino - 1) & 1);  // the previous item's dQ is stored
+          tc_fence_after();
+          // dS of keys [64u, 64u+64) sits in columns 64u .. 64u+31 of the dP range
+          const uint32_t kt_lo = kt_lo0 + st * (C::kStage >> 4);
 #pragma unroll
-        for (int k = 0; k < kBN / 16; ++k)
-          umma_ts_lo(tmem + C::kdQ, tmem + C::kdP + (k >> 2) * 64 + (k & 3) * 8,
-                     kt_lo + mnmajor_step(k), idesc_dq, (j > 0 || k > 0));
-        tc_commit(bar_e + st);
-        if (j + 1 < n_tiles) issue_dp(j + 1);
+          for (int k = 0; k < kBN / 16; ++k)
+            umma_ts_lo(tmem + C::kdQ, tmem + C::kdP + (k >> 2) * 64 + (k & 3) * 8,
+                       kt_lo + mnmajor_step(k), idesc_dq, (j > 0 || k > 0));
+          tc_commit(bar_e + st);
+          if (j + 1 < n_tiles) issue_dp(gi + 1);
+        }
+        tc_commit(bar_acc);
+        tb += n_tiles;
       }
-      tc_commit(bar_acc);
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
     const int u = (warp >= 8) ? 1 : 0;
     const int r = tid & 127;
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-    const int row = t * kBM + r;
-    const bool row_ok = row < p.L;
-    // ---------------- Q (warps 4-7) and dO (warps 8-11) rows into tensor memory ----------------
-    {
+    const uint32_t tS = tmem + lane_base + C::kS + u * 64;
+    const uint32_t tdP = tmem + lane_base + C::kdP + u * 64;
+    // Q (warps 4-7) or dO (warps 8-11) row of an item into tensor memory
+    auto load_qdo = [&](const DqItem& it) {
+      const int row = it.t * kBM + r;
+      const bool row_ok = row < p.L;
       const uint4* src = reinterpret_cast<const uint4*>((u ? dOg : Qg) +
-                                                        (size_t(q_plane) * p.L + row) * D);
+                                                        (size_t(it.q_plane) * p.L + row) * D);
       const uint32_t dst = tmem + lane_base + (u ? C::kdOt : C::kQt);
 #pragma unroll
       for (int c = 0; c < D / 64; ++c) {
@@ -267,88 +299,103 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive_warp(bar_qdo);
-    }
-    // ---------------- dS: warpgroup u takes key columns [64u, 64u+64) of every tile -----------
-    const uint32_t tS = tmem + lane_base + C::kS + u * 64;
-    const uint32_t tdP = tmem + lane_base + C::kdP + u * 64;
-    const int lim_i = row_ok ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-    const float2 stt = row_ok ? p.stats[size_t(q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
-    const float neg_lse2 = -stt.x, delta_i = stt.y;
-    for (int j = 0; j < n_tiles; ++j) {
-      const bool side = j < ns;
-      int c_lo = 0, c_hi = kBN;
-      bool need_mask;
-      if (side) {
-        c_hi = lim_i - j * kBN;
-        need_mask = (j >= g.side_full);
-      } else {
-        const int key0 = tile_y(j);
-        c_hi = row - key0 + 1;
-        c_lo = row - p.n_neighbor + 1 - key0;
-        need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-      }
-      // phase A (needs S only; runs under the previous tile's dQ and this tile's dP MMAs):
-      // P = exp2(S * scale - LSE), kept in registers
-      wait(bar_s, j & 1);
-      tc_fence_after();
-      uint32_t sv[2][32];
-      tmem_ld32(tS, sv[0]);
-      tmem_ld32(tS + 32, sv[1]);
-      tmem_ld_wait();
-      tc_fence_before();
-      mbar_arrive_warp(bar_sl);  // the S columns may be overwritten from here on
-      if (need_mask) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int col = u * 64 + c * 32 + e;
-            const float pr = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
-            sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? pr : 0.f);
-          }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2)));
-      }
-      // phase B: dS = P (dP - Delta)
-      wait(bar_dp, j & 1);
-      tc_fence_after();
-      uint32_t pk[32];
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t dp[32];
-        tmem_ld32(tdP + c * 32, dp);
+    };
+    int tb = 0, ino = 0;
+    if (int(blockIdx.x) < n_items) load_qdo(dq_item(p, blockIdx.x));
+    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++ino) {
+      const DqItem it = dq_item(p, w);
+      const int t = it.t, ns = it.ns;
+      const int row = t * kBM + r;
+      const bool row_ok = row < p.L;
+      // ---------------- dS: warpgroup u takes key columns [64u, 64u+64) of every tile ---------
+      const int lim_i = row_ok ? min(p.lim[size_t(it.b) * p.L + row], p.side_cap) : 0;
+      const float2 stt = row_ok ? p.stats[size_t(it.q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
+      const float neg_lse2 = -stt.x, delta_i = stt.y;
+      for (int j = 0; j < it.n_tiles; ++j) {
+        const int gi = tb + j;
+        const bool side = j < ns;
+        int c_lo = 0, c_hi = kBN;
+        bool need_mask;
+        if (side) {
+          c_hi = lim_i - j * kBN;
+          need_mask = (j >= it.side_full);
+        } else {
+          const int key0 = (it.wlo + (j - ns)) * kBN;
+          c_hi = row - key0 + 1;
+          c_lo = row - p.n_neighbor + 1 - key0;
+          need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
+        }
+        // phase A (needs S only; runs under the previous tile's dQ and this tile's dP MMAs):
+        // P = exp2(S * scale - LSE), kept in registers
+        wait(bar_s, gi & 1);
+        tc_fence_after();
+        uint32_t sv[2][32];
+        tmem_ld32(tS, sv[0]);
+        tmem_ld32(tS + 32, sv[1]);
         tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive_warp(bar_sl);  // the S columns may be overwritten from here on
+        if (need_mask) {
 #pragma unroll
-        for (int e = 0; e < 32; e += 2)
-          pk[c * 16 + (e >> 1)] =
-              pack_bf16(__uint_as_float(sv[c][e]) * (__uint_as_float(dp[e]) - delta_i),
-                        __uint_as_float(sv[c][e + 1]) * (__uint_as_float(dp[e + 1]) - delta_i));
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int col = u * 64 + c * 32 + e;
+              const float pr = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
+              sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? pr : 0.f);
+            }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2)));
+        }
+        // phase B: dS = P (dP - Delta)
+        wait(bar_dp, gi & 1);
+        tc_fence_after();
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t dp[32];
+          tmem_ld32(tdP + c * 32, dp);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2)
+            pk[c * 16 + (e >> 1)] =
+                pack_bf16(__uint_as_float(sv[c][e]) * (__uint_as_float(dp[e]) - delta_i),
+                          __uint_as_float(sv[c][e + 1]) * (__uint_as_float(dp[e + 1]) - delta_i));
+        }
+        // packed dS over the first half of this thread's own dP columns
+        tmem_st32(tdP, pk);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive_warp(bar_ds);
       }
-      // packed dS over the first half of this thread's own dP columns
-      tmem_st32(tdP, pk);
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive_warp(bar_ds);
-    }
-    // ---------------- epilogue: each warpgroup stores half of the row ----------------
-    wait(bar_acc, 0);
-    tc_fence_after();
-    const uint32_t t_acc = tmem + lane_base + C::kdQ + u * (D / 2);
+      tb += it.n_tiles;
+      // Every S and dP MMA of this item is complete (the last dP was waited for), so Q and dO of
+      // the next item can go into tensor memory while this item's last dQ MMAs run.
+      if (w + int(gridDim.x) < n_items) load_qdo(dq_item(p, w + gridDim.x));
+      // ---------------- epilogue: each warpgroup stores half of the row ----------------
+      wait(bar_acc, ino & 1);
+      tc_fence_after();
+      const uint32_t t_acc = tmem + lane_base + C::kdQ + u * (D / 2);
 #pragma unroll
-    for (int c = 0; c < D / 64; ++c) {
-      uint32_t rr[32];
-      tmem_ld32(t_acc + c * 32, rr);
-      tmem_ld_wait();
-      if (row_ok) {
-        float v[32];
+      for (int c = 0; c < D / 64; ++c) {
+        uint32_t rr[32];
+        tmem_ld32(t_acc + c * 32, rr);
+        tmem_ld_wait();
+        if (c == D / 64 - 1) {  // dQ is in registers: the next item may start accumulating
+          tc_fence_before();
+          mbar_arrive_warp(bar_dqf);
+        }
+        if (row_ok) {
+          float v[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
-        store_row_chunk32(p.dQ, (size_t(q_plane) * p.L + row) * D + u * (D / 2) + c * 32,
-                          p.grad_fp32, v);
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
+          store_row_chunk32(p.dQ, (size_t(it.q_plane) * p.L + row) * D + u * (D / 2) + c * 32,
+                            p.grad_fp32, v);
+        }
       }
     }
   }
@@ -807,9 +854,12 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        int(DkvCfg<D>::kRequest)));
-  bwd_dq_kernel<D><<<dim3(d->Hq * d->B, ih.n_tiles), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
-      mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q),
-      static_cast<const __nv_bfloat16*>(dO), p);
+  {
+    const int n_items = d->Hq * d->B * ih.n_tiles;
+    bwd_dq_kernel<D><<<std::min(n_items, sm_count()), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
+        mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO),
+        p, n_items);
+  }
   record_event(d, 3, stream);
   bwd_dkv_kernel<D, true><<<dim3(d->Hkv * lay.split * d->B, lay.cap_pad / kBN), kBwdThreads,
                             DkvCfg<D>::kRequest, stream>>>(mq, mdo, mks, mvs, p);

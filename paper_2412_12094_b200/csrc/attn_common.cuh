@@ -57,6 +57,15 @@ __global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
                                int cap_pad, __nv_bfloat16* __restrict__ Ks,
                                __nv_bfloat16* __restrict__ Vs);
 
+// Number of SMs of the current device (persistent kernels launch one CTA per SM).
+inline int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+    return 148;
+  return n;
+}
+
 // Records desc->events[i] on the stream if the caller asked for it.
 inline void record_event(const sepllm_attn_desc* d, int i, cudaStream_t stream) {
   if (d->events && i < d->n_events && d->events[i])

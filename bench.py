@@ -295,7 +295,7 @@ def bench_decode(device, peaks, steps=4096):
                 size_sep[b] = min(c["s"], size_sep[b] + sum(win_flags[b][:n_past]))
                 win_flags[b] = win_flags[b][n_past:]
             rows += size_init[b] + size_sep[b] + len(win_flags[b])
-    # One CUDA graph holds `pool` consecutive steps (4 kernels each); the token ids of a chunk are
+    # One CUDA graph holds `pool` consecutive steps (3 kernels each); the token ids of a chunk are
     # copied into the graph's fixed input buffer inside the timed region.
     assert warm % pool == 0 and steps % pool == 0
     ids_buf = torch.empty((pool, B), dtype=torch.int32, device=device)
@@ -327,7 +327,7 @@ def bench_decode(device, peaks, steps=4096):
             "bytes_per_step": bytes_total / steps, "achieved_gbs": gbs,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "traffic": None},
-            "tokens_per_s": B * steps / sec, "gpu_launches": 4 * steps}
+            "tokens_per_s": B * steps / sec, "gpu_launches": 3 * steps}
 
 
 def bench_index_stream(device, peaks, reps=20):

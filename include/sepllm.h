@@ -198,7 +198,8 @@ typedef struct {
   int64_t reserved[22];
 } sepllm_cache_header; /* 256 bytes */
 
-/* Per-sequence record inside the state, 16 int32. */
+/* Per-sequence record inside the state, 16 int32.  reserved[0] is a scratch
+ * counter of sepllm_cache_update (zero between calls); the rest is zero. */
 typedef struct {
   int32_t size_init, sep_start, size_sep, win_start, size_win, compactions;
   int64_t next_pos;              /* tokens seen so far */

@@ -123,16 +123,22 @@ __device__ int rank_past_separators(const uint8_t* slot_is_sep_b, const sepllm_c
 
 constexpr int kMaxPast = 24576;  // int16 ranks in shared memory: 48 KB
 
-// grid (B, Hkv): K/V movement for one kv head of one sequence.  Reads the state, never writes it.
+// grid (B, Hkv).  Every CTA moves the K/V rows of its kv head (append; at a compaction the ordered
+// move of Past-Window separators into the separator ring), reading the sequence's state only.
+// The CTA that finishes last for a sequence (an arrival count in the sequence record) then
+// updates the per-slot metadata and the record, so the state changes only after every kv head
+// has planned its moves from the old one -- one launch instead of two.
 __global__ void __launch_bounds__(kUpdThreads)
-cache_update_kv(sepllm_cache_header h, const uint8_t* __restrict__ state,
-                __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc,
-                const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new) {
+cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* __restrict__ Kc,
+             __nv_bfloat16* __restrict__ Vc, const __nv_bfloat16* __restrict__ k_new,
+             const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ new_token_ids,
+             SepIds sep) {
   extern __shared__ int16_t flag_s[];
   __shared__ int warp_buf[32];
+  __shared__ int s_last;
   const sepllm_cache_desc d = h.desc;
   const int b = blockIdx.x, hk = blockIdx.y, tid = threadIdx.x;
-  CacheView v = cache_view(const_cast<uint8_t*>(state), h);
+  CacheView v = cache_view(state, h);
   const sepllm_cache_seq q = v.seq[b];
   const UpdatePlan p = plan_update(q, d);
   const size_t plane = (size_t(b) * d.Hkv + hk) * h.slots * d.d;
@@ -143,58 +149,52 @@ cache_update_kv(sepllm_cache_header h, const uint8_t* __restrict__ state,
   const uint4* vn = reinterpret_cast<const uint4*>(v_new + (size_t(b) * d.Hkv + hk) * d.d);
   if (tid < vec) Kp[size_t(p.append_slot) * vec + tid] = kn[tid];
   else if (tid < 2 * vec) Vp[size_t(p.append_slot) * vec + (tid - vec)] = vn[tid - vec];
-  if (!p.compact || d.s == 0) return;
 
-  const int m = rank_past_separators(v.slot_is_sep + size_t(b) * h.slots, q, d, p.n_past, flag_s,
-                                     warp_buf);
-  const int drop = max(0, q.size_sep + m - d.s);
+  const bool moves = p.compact && d.s > 0;  // the same for every thread of the block
   const int ring = d.c - d.a, wbase = d.a + d.s;
-  // one half-warp (16 lanes x 16 bytes = 256 bytes) moves a K row, the other the V row when d=128;
-  // generic: `vec` lanes per row
-  const int rows_per_pass = kUpdThreads / (2 * vec);
-  const int sub = tid / (2 * vec), l = tid % (2 * vec);
-  for (int k = sub; k < p.n_past; k += rows_per_pass) {
-    const int r = flag_s[k];
-    if (r == 0) continue;
-    const int fifo = q.size_sep + (r - 1);  // place in the queue of old + moved separators
-    if (fifo < drop) continue;              // falls out at once
-    const int src = wbase + (q.win_start + k) % ring;
-    const int dst = d.a + (q.sep_start + fifo) % d.s;
-    if (l < vec) Kp[size_t(dst) * vec + l] = Kp[size_t(src) * vec + l];
-    else Vp[size_t(dst) * vec + (l - vec)] = Vp[size_t(src) * vec + (l - vec)];
+  int m = 0, drop = 0;
+  if (moves) {
+    m = rank_past_separators(v.slot_is_sep + size_t(b) * h.slots, q, d, p.n_past, flag_s, warp_buf);
+    drop = max(0, q.size_sep + m - d.s);
+    // `vec` lanes move a K row, the next `vec` lanes the V row
+    const int rows_per_pass = kUpdThreads / (2 * vec);
+    const int sub = tid / (2 * vec), l = tid % (2 * vec);
+    for (int k = sub; k < p.n_past; k += rows_per_pass) {
+      const int r = flag_s[k];
+      if (r == 0) continue;
+      const int fifo = q.size_sep + (r - 1);  // place in the queue of old + moved separators
+      if (fifo < drop) continue;              // falls out at once
+      const int src = wbase + (q.win_start + k) % ring;
+      const int dst = d.a + (q.sep_start + fifo) % d.s;
+      if (l < vec) Kp[size_t(dst) * vec + l] = Kp[size_t(src) * vec + l];
+      else Vp[size_t(dst) * vec + (l - vec)] = Vp[size_t(src) * vec + (l - vec)];
+    }
   }
-}
 
-// grid (B): per-slot metadata and the sequence record.  Runs after cache_update_kv.
-__global__ void __launch_bounds__(kUpdThreads)
-cache_update_state(sepllm_cache_header h, uint8_t* __restrict__ state,
-                   const int32_t* __restrict__ new_token_ids, SepIds sep) {
-  extern __shared__ int16_t flag_s[];
-  __shared__ int warp_buf[32];
-  const sepllm_cache_desc d = h.desc;
-  const int b = blockIdx.x, tid = threadIdx.x;
-  CacheView v = cache_view(state, h);
-  const sepllm_cache_seq q = v.seq[b];
-  const UpdatePlan p = plan_update(q, d);
+  // last kv head of the sequence to get here updates the state
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const int prev = atomicAdd(&v.seq[b].reserved[0], 1);
+    s_last = (prev == d.Hkv - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
   int64_t* pos_b = v.slot_pos + size_t(b) * h.slots;
   uint8_t* sep_b = v.slot_is_sep + size_t(b) * h.slots;
-  const bool f = is_separator(new_token_ids[b], sep);
-  __syncthreads();  // every thread holds the old record before it changes
   if (tid == 0) {
     pos_b[p.append_slot] = q.next_pos;
-    sep_b[p.append_slot] = uint8_t(f);
+    sep_b[p.append_slot] = uint8_t(is_separator(new_token_ids[b], sep));
   }
   sepllm_cache_seq nq = q;
+  nq.reserved[0] = 0;  // arrival count for the next update
   nq.next_pos = q.next_pos + 1;
   if (q.size_init < d.a) nq.size_init = q.size_init + 1;
   else nq.size_win = q.size_win + 1;
-
   if (p.compact) {
-    int m = 0, drop = 0;
-    if (d.s > 0) {
-      m = rank_past_separators(sep_b, q, d, p.n_past, flag_s, warp_buf);
-      drop = max(0, q.size_sep + m - d.s);
-      const int ring = d.c - d.a, wbase = d.a + d.s;
+    if (moves) {
       for (int k = tid; k < p.n_past; k += kUpdThreads) {
         const int r = flag_s[k];
         if (r == 0) continue;
@@ -208,7 +208,7 @@ cache_update_state(sepllm_cache_header h, uint8_t* __restrict__ state,
       nq.sep_start = (q.sep_start + drop) % d.s;
       nq.size_sep = q.size_sep + m - drop;
     }
-    nq.win_start = (q.win_start + p.n_past) % (d.c - d.a);
+    nq.win_start = (q.win_start + p.n_past) % ring;
     nq.size_win = d.w;
     nq.compactions = q.compactions + 1;
   }
@@ -546,18 +546,13 @@ extern "C" sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void
   sep.n = n_sep;
   for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k) sep.id[k] = (k < n_sep) ? sep_ids[k] : -1;
   const size_t smem = size_t(max_past) * sizeof(int16_t);
-  if (smem > 40 * 1024) {
-    SEPLLM_CUDA_TRY(cudaFuncSetAttribute(cache_update_kv,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    SEPLLM_CUDA_TRY(cudaFuncSetAttribute(cache_update_state,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-  }
-  cache_update_kv<<<dim3(desc->B, desc->Hkv), kUpdThreads, smem, stream>>>(
-      h, static_cast<const uint8_t*>(state), static_cast<__nv_bfloat16*>(Kc),
+  if (smem > 40 * 1024)
+    SEPLLM_CUDA_TRY(cudaFuncSetAttribute(cache_update, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         int(smem)));
+  cache_update<<<dim3(desc->B, desc->Hkv), kUpdThreads, smem, stream>>>(
+      h, static_cast<uint8_t*>(state), static_cast<__nv_bfloat16*>(Kc),
       static_cast<__nv_bfloat16*>(Vc), static_cast<const __nv_bfloat16*>(k_new),
-      static_cast<const __nv_bfloat16*>(v_new));
-  cache_update_state<<<desc->B, kUpdThreads, smem, stream>>>(h, static_cast<uint8_t*>(state),
-                                                            new_token_ids, sep);
+      static_cast<const __nv_bfloat16*>(v_new), new_token_ids, sep);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }

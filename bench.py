@@ -250,8 +250,9 @@ def kernel_times(wl: Workload, steps: int):
     }
 
 
-def bench_decode(device, peaks, steps=4096):
-    """Streaming workload: cache update + decode per step at the full cache shape."""
+def bench_decode(device, peaks, steps=4096, rope=False):
+    """Streaming workload: cache update + decode per step at the full cache shape.  rope: decode
+    with positions inside the cache (K cached un-rotated, rotated on the fly)."""
     from paper_2412_12094_b200 import api
     c = inputs.DECODE_CONFIG
     B, Hq, Hkv, d = c["B"], c["Hq"], c["Hkv"], c["d"]
@@ -262,6 +263,9 @@ def bench_decode(device, peaks, steps=4096):
     Vc = torch.zeros(kb // 2, dtype=torch.bfloat16, device=device)
     ws = api.alloc_bytes(api.sepllm_decode_workspace_bytes(desc))
     api.sepllm_cache_init(desc, state)
+    if rope:
+        table = api.alloc_bytes(api.sepllm_rope_table_bytes(desc))
+        api.sepllm_rope_table_build(desc, 500000.0, table)
     pool = 256
     warm = 12032                      # enough tokens to fill the separator cache (s / rho plus slack)
     T = warm + steps
@@ -273,7 +277,10 @@ def bench_decode(device, peaks, steps=4096):
 
     def step(t, ids_row):
         api.sepllm_cache_update(desc, state, Kc, Vc, ids_row, inputs.SEP_IDS, kp[t % pool], vp[t % pool])
-        api.sepllm_decode(desc, 0.0, qp[t % pool], state, Kc, Vc, o, lse, ws)
+        if rope:
+            api.sepllm_decode_rope(desc, 0.0, qp[t % pool], state, Kc, Vc, table, o, lse, ws)
+        else:
+            api.sepllm_decode(desc, 0.0, qp[t % pool], state, Kc, Vc, o, lse, ws)
 
     for t in range(warm):
         step(t, ids_d[t])
@@ -322,7 +329,8 @@ def bench_decode(device, peaks, steps=4096):
     sec = e0.elapsed_time(e1) / 1e3
     bytes_total = rows * Hkv * d * 2 * 2          # K and V rows of every retained entry, every kv head
     gbs = bytes_total / sec / 1e9
-    return {"workload": "B32 Hq32 Hkv8 d128 a4 s1024 w256 c3332, update+decode per step",
+    return {"workload": "B32 Hq32 Hkv8 d128 a4 s1024 w256 c3332, update+decode per step"
+                        + (", rotary positions inside the cache (base 500000)" if rope else ""),
             "steps": steps, "us_per_step": sec / steps * 1e6, "avg_size_run": rows / steps / B,
             "bytes_per_step": bytes_total / steps, "achieved_gbs": gbs,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -365,7 +373,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_long_r10", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / index-stream / e2e / CPU legs")
-    ap.add_argument("--leg", default="all", choices=["all", "decode", "index"],
+    ap.add_argument("--leg", default="all", choices=["all", "decode", "decode_rope", "index"],
                     help="decode / index: run only that secondary leg and print its JSON")
     ap.add_argument("--cpu-prefix", type=int, default=8192)
     ap.add_argument("--cpu-heads", type=int, default=4)
@@ -420,7 +428,8 @@ def main():
 
     peaks = load_peaks()
     if args.leg != "all":
-        print(json.dumps(bench_decode(device, peaks) if args.leg == "decode" else bench_index_stream(device, peaks)))
+        print(json.dumps(bench_index_stream(device, peaks) if args.leg == "index"
+                         else bench_decode(device, peaks, rope=(args.leg == "decode_rope"))))
         return
     wl = Workload(args.workload, rank, device)
     wl.step()
@@ -475,6 +484,7 @@ def main():
             del wl
             torch.cuda.empty_cache()
             out["decode"] = bench_decode(device, peaks)
+            out["decode_rope"] = bench_decode(device, peaks, rope=True)
             out["index"] = bench_index_stream(device, peaks)
             if world == 1:
                 v, dt, cores, what = oracle_sample(cfg, args.cpu_heads, args.cpu_prefix)

@@ -233,6 +233,28 @@ sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const vo
                             const void* state, const void* Kc, const void* Vc, void* o,
                             float* lse, void* workspace, void* stream);
 
+/* Decode with positions taken inside the cache (Section 3.3, "Positional
+ * Encoding": as in StreamingLLM, the streaming setting uses an entry's place in
+ * the cache, not its place in the text; Table 8 shows the effect of leaving
+ * this out).  K is cached un-rotated and q is passed un-rotated; the retained
+ * entries, walked as initial, separator (oldest first), neighbour (oldest
+ * first), get positions 0 .. Size_run-1 and the query gets Size_run-1.  The
+ * paper fixes no rotary formula; this library uses the rotate-half form:
+ * with theta_i = base^(-2i/d), i < d/2, a vector x at position p becomes
+ *   y[i]       = x[i] cos(p theta_i) - x[i + d/2] sin(p theta_i)
+ *   y[i + d/2] = x[i + d/2] cos(p theta_i) + x[i] sin(p theta_i).
+ * rope_table holds (cos, sin) as fp32 pairs [c][d/2]: size it with
+ * sepllm_rope_table_bytes and fill it once per (desc, base) with
+ * sepllm_rope_table_build (dev, 16-byte aligned).  Rotated K and q are
+ * rounded to bf16 before the products.  Other arguments as sepllm_decode. */
+sepllm_status sepllm_rope_table_bytes(const sepllm_cache_desc* desc, size_t* bytes);
+sepllm_status sepllm_rope_table_build(const sepllm_cache_desc* desc, float rope_base, void* table,
+                                      void* stream);
+sepllm_status sepllm_decode_rope(const sepllm_cache_desc* desc, float scale, const void* q,
+                                 const void* state, const void* Kc, const void* Vc,
+                                 const void* rope_table, void* o, float* lse, void* workspace,
+                                 void* stream);
+
 /* Copies the device status word at the start of an index, workspace or state
  * buffer to *out (host) after synchronising `stream`. */
 sepllm_status sepllm_last_device_status(const void* buffer, int32_t* out, void* stream);

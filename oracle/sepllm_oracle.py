@@ -417,3 +417,32 @@ def decode_attention(q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, scale: float
     e = np.exp(lam - mx)
     Z = e.sum()
     return (e / Z) @ Vc, mx + math.log(Z)
+
+
+# ----------------------------------------------------------------------------
+# Decode with positions inside the cache (Section 3.3, "Positional Encoding")
+# ----------------------------------------------------------------------------
+
+def rope_rotate(x: np.ndarray, pos, base: float) -> np.ndarray:
+    """Rotary encoding, rotate-half form (the paper names no formula; this is
+    the library's stated reading).  x [..., d]; pos broadcastable to x[..., 0].
+    theta_i = base^(-2i/d); (x_i, x_{i+d/2}) turns by the angle pos * theta_i."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    h = d // 2
+    theta = base ** (-2.0 * np.arange(h) / d)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * theta
+    c, s = np.cos(ang), np.sin(ang)
+    lo, hi = x[..., :h], x[..., h:]
+    return np.concatenate([lo * c - hi * s, hi * c + lo * s], axis=-1)
+
+
+def decode_attention_rope(q, Kc, Vc, base: float, q_pos=None, k_pos=None, scale: float | None = None):
+    """One un-rotated query over un-rotated retained keys given in cache order:
+    key r sits at position r and the query at position R-1 (positions within
+    the cache, not in the text), unless positions are passed explicitly."""
+    Kc = np.asarray(Kc, dtype=np.float64)
+    R = Kc.shape[0]
+    k_pos = np.arange(R) if k_pos is None else np.asarray(k_pos)
+    q_pos = R - 1 if q_pos is None else q_pos
+    return decode_attention(rope_rotate(q, np.asarray(q_pos), base), rope_rotate(Kc, k_pos, base), Vc, scale)

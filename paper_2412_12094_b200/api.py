@@ -65,7 +65,8 @@ EXPORTS = [
     "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_static",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
-    "sepllm_decode_workspace_bytes", "sepllm_decode", "sepllm_last_device_status",
+    "sepllm_decode_workspace_bytes", "sepllm_decode", "sepllm_rope_table_bytes",
+    "sepllm_rope_table_build", "sepllm_decode_rope", "sepllm_last_device_status",
     "sepllm_status_string",
 ]
 
@@ -212,6 +213,23 @@ def sepllm_decode_workspace_bytes(desc):
 def sepllm_decode(desc, scale, q, state, Kc, Vc, o, lse, workspace):
     _check(lib().sepllm_decode(C.byref(desc), C.c_float(scale), _ptr(q), _ptr(state), _ptr(Kc), _ptr(Vc),
                                _ptr(o), _ptr(lse), _ptr(workspace), _stream()), "sepllm_decode")
+
+
+def sepllm_rope_table_bytes(desc):
+    b = C.c_size_t(0)
+    _check(lib().sepllm_rope_table_bytes(C.byref(desc), C.byref(b)), "sepllm_rope_table_bytes")
+    return b.value
+
+
+def sepllm_rope_table_build(desc, rope_base, table):
+    _check(lib().sepllm_rope_table_build(C.byref(desc), C.c_float(rope_base), _ptr(table), _stream()),
+           "sepllm_rope_table_build")
+
+
+def sepllm_decode_rope(desc, scale, q, state, Kc, Vc, rope_table, o, lse, workspace):
+    _check(lib().sepllm_decode_rope(C.byref(desc), C.c_float(scale), _ptr(q), _ptr(state), _ptr(Kc),
+                                    _ptr(Vc), _ptr(rope_table), _ptr(o), _ptr(lse), _ptr(workspace),
+                                    _stream()), "sepllm_decode_rope")
 
 
 def read_cache_state(state: torch.Tensor) -> dict:

@@ -281,12 +281,17 @@ constexpr int decode_smem_bytes() {
 // dimension of warp-level MMAs (rows G..15 are zero), scores go through an online softmax with a
 // lazily moved reference, and O accumulates in registers.  The four warps' partials are merged
 // through shared memory into one (m, l, acc) record per (query head, split).
-template <int D>
+//
+// ROPE: K rows are cached un-rotated and q arrives un-rotated; positions are indices within the
+// cache (entry v of the walk above sits at position v, the query at Size_run - 1).  Each warp
+// rotates its K tile in shared memory, pair (i, i + D/2) by the angle v * theta_i, from a table of
+// (cos, sin) per (position, i), before the MMAs read it; q is rotated while its fragments load.
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
              const uint8_t* __restrict__ state, const __nv_bfloat16* __restrict__ Kc,
              const __nv_bfloat16* __restrict__ Vc, float* __restrict__ part_ml,
-             float* __restrict__ part_acc, int splits) {
+             float* __restrict__ part_acc, int splits, const float2* __restrict__ rope) {
   constexpr int CH = D / 8;                 // 16-byte chunks per row
   constexpr int ROWB = D * 2;               // bytes per row
   constexpr int TILEB = kDecTile * ROWB;    // bytes of one K (or V) tile
@@ -316,10 +321,21 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   uint32_t qa[D / 16][4];
   {
     const __nv_bfloat16* qrow = q_in + (size_t(b) * d.Hq + hk * G + min(frow, G - 1)) * D;
+    // two consecutive elements e, e+1 of the (rotated) query row as packed bf16
+    auto q_pair = [&](int e) -> uint32_t {
+      if (!ROPE) return *reinterpret_cast<const uint32_t*>(qrow + e);
+      const int i = e % (D / 2);
+      const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qrow + e));
+      const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qrow + (e ^ (D / 2))));
+      const float2 cs0 = rope[size_t(size_run - 1) * (D / 2) + i];
+      const float2 cs1 = rope[size_t(size_run - 1) * (D / 2) + i + 1];
+      const float sgn = (e < D / 2) ? -1.f : 1.f;  // first half: x cos - y sin; second: x cos + y sin
+      return pack_bf16(x.x * cs0.x + sgn * y.x * cs0.y, x.y * cs1.x + sgn * y.y * cs1.y);
+    };
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-      qa[ks][0] = (frow < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + fcol) : 0u;
-      qa[ks][2] = (frow < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + fcol) : 0u;
+      qa[ks][0] = (frow < G && size_run > 0) ? q_pair(ks * 16 + fcol) : 0u;
+      qa[ks][2] = (frow < G && size_run > 0) ? q_pair(ks * 16 + 8 + fcol) : 0u;
       qa[ks][1] = 0u;
       qa[ks][3] = 0u;
     }
@@ -363,6 +379,32 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
     cp_async_commit();
 
     const uint32_t sK = wbase_u + (i % kDecStages) * 2 * TILEB, sV = sK + TILEB;
+    if (ROPE) {
+      // rotate the tile's K rows in place: a lane takes (row, 8 pairs) items; the two 16-byte
+      // chunks of a pair group are chunk c (elements 8c..8c+7) and chunk c + CH/2
+      uint8_t* tK = wbase + (i % kDecStages) * 2 * TILEB;
+      const int vrow0 = v0 + (wid + i * NW) * kDecTile;
+      for (int item = lane; item < kDecTile * (CH / 2); item += 32) {
+        const int r = item / (CH / 2), c = item % (CH / 2);
+        uint4* plo = reinterpret_cast<uint4*>(tK + r * ROWB + ((c ^ (r & 7)) << 4));
+        uint4* phi = reinterpret_cast<uint4*>(tK + r * ROWB + (((c + CH / 2) ^ (r & 7)) << 4));
+        uint4 lo = *plo, hi = *phi;
+        const float4* cs = reinterpret_cast<const float4*>(
+            rope + size_t(min(vrow0 + r, size_run - 1)) * (D / 2) + c * 8);
+        __nv_bfloat162* lo2 = reinterpret_cast<__nv_bfloat162*>(&lo);
+        __nv_bfloat162* hi2 = reinterpret_cast<__nv_bfloat162*>(&hi);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float4 t4 = cs[e];  // (cos, sin) of pairs 2e and 2e+1
+          const float2 x = __bfloat1622float2(lo2[e]), y = __bfloat1622float2(hi2[e]);
+          lo2[e] = __floats2bfloat162_rn(x.x * t4.x - y.x * t4.y, x.y * t4.z - y.y * t4.w);
+          hi2[e] = __floats2bfloat162_rn(y.x * t4.x + x.x * t4.y, y.y * t4.z + x.y * t4.w);
+        }
+        *plo = lo;
+        *phi = hi;
+      }
+      __syncwarp();
+    }
     // S[16 heads x 16 rows] = Q K^T
     float sc[2][4];
 #pragma unroll
@@ -483,6 +525,19 @@ __global__ void decode_combine(sepllm_cache_header h, const float* __restrict__ 
   if (lse && e == 0) lse[row] = (ll > 0.f) ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
 }
 
+// (cos, sin) of position * base^(-2i/D) for every position a cache entry can have and every
+// pair index i < D/2.
+__global__ void rope_table_kernel(float2* __restrict__ table, int positions, int half_d,
+                                  float log2_base) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= positions * half_d) return;
+  const int pos = idx / half_d, i = idx % half_d;
+  const float theta = exp2f(-log2_base * float(i) / float(half_d));
+  float sn, cs;
+  sincosf(float(pos) * theta, &sn, &cs);
+  table[idx] = make_float2(cs, sn);
+}
+
 static int decode_splits(const sepllm_cache_desc* d) {
   // about four CTAs per SM over the whole grid, each with at least 256 rows (64 per warp)
   const int units = d->B * d->Hkv;
@@ -568,23 +623,25 @@ extern "C" sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* 
   return SEPLLM_OK;
 }
 
-template <int D>
+template <int D, bool ROPE>
 static sepllm_status launch_decode(const sepllm_cache_header& h, float scale_log2, const void* q,
                                    const void* state, const void* Kc, const void* Vc, float* ml,
-                                   float* acc, int splits, cudaStream_t stream) {
+                                   float* acc, int splits, const float2* rope, cudaStream_t stream) {
   constexpr int smem = decode_smem_bytes<D>();
   static_assert(smem >= (kDecThreads / 32) * 8 * (8 + D * 4), "partials fit in the stage buffers");
-  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       smem));
-  decode_split<D><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D, ROPE>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  decode_split<D, ROPE><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
       h, scale_log2, static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(state),
-      static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc, splits);
+      static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc, splits,
+      rope);
   return SEPLLM_OK;
 }
 
-extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const void* q,
-                                       const void* state, const void* Kc, const void* Vc, void* o,
-                                       float* lse, void* workspace, void* stream_) {
+static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, const void* q,
+                                 const void* state, const void* Kc, const void* Vc,
+                                 const float2* rope, void* o, float* lse, void* workspace,
+                                 void* stream_) {
   sepllm_cache_header h;
   sepllm_status st = fill_cache_header(desc, &h);
   if (st != SEPLLM_OK) return st;
@@ -602,9 +659,11 @@ extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scal
   if (scale == 0.f) scale = 1.0f / sqrtf(float(desc->d));
   const float scale_log2 = scale * 1.4426950408889634f;
   if (desc->d == 128)
-    st = launch_decode<128>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, stream);
+    st = rope ? launch_decode<128, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
+              : launch_decode<128, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
   else
-    st = launch_decode<64>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, stream);
+    st = rope ? launch_decode<64, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
+              : launch_decode<64, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
   if (st != SEPLLM_OK) return st;
   if (desc->d == 128)
     decode_combine<128><<<dim3(desc->Hq, desc->B), 128, 0, stream>>>(
@@ -614,4 +673,40 @@ extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scal
         h, ml, acc, splits, static_cast<__nv_bfloat16*>(o), lse);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const void* q,
+                                       const void* state, const void* Kc, const void* Vc, void* o,
+                                       float* lse, void* workspace, void* stream_) {
+  return decode_impl(desc, scale, q, state, Kc, Vc, nullptr, o, lse, workspace, stream_);
+}
+
+extern "C" sepllm_status sepllm_rope_table_bytes(const sepllm_cache_desc* desc, size_t* bytes) {
+  sepllm_cache_header h;
+  sepllm_status st = fill_cache_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  if (bytes) *bytes = align_up(size_t(desc->c) * (desc->d / 2) * sizeof(float2));
+  return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_rope_table_build(const sepllm_cache_desc* desc, float rope_base,
+                                                 void* table, void* stream_) {
+  sepllm_cache_header h;
+  sepllm_status st = fill_cache_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  if (!table || !aligned(table, 16) || !(rope_base > 1.f)) return SEPLLM_INVALID_ARG;
+  const int n = desc->c * (desc->d / 2);
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream_)>>>(
+      static_cast<float2*>(table), desc->c, desc->d / 2, log2f(rope_base));
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_decode_rope(const sepllm_cache_desc* desc, float scale,
+                                            const void* q, const void* state, const void* Kc,
+                                            const void* Vc, const void* rope_table, void* o,
+                                            float* lse, void* workspace, void* stream_) {
+  if (!rope_table || !aligned(rope_table, 16)) return SEPLLM_INVALID_ARG;
+  return decode_impl(desc, scale, q, state, Kc, Vc, static_cast<const float2*>(rope_table), o, lse,
+                     workspace, stream_);
 }

@@ -308,3 +308,31 @@ def test_selected_key_gradients_equal_the_all_rows_backward():
     gk, gv = orc.attn_keys_bwd(Q, K, V, dO, f, a, n, keys)
     assert np.allclose(gk, dK[keys], rtol=1e-12, atol=1e-12)
     assert np.allclose(gv, dV[keys], rtol=1e-12, atol=1e-12)
+
+
+def test_rope_decode_pins():
+    """The rotary decode of the oracle against what the mathematics fixes: rotation as complex
+    multiplication (an independent formulation), norm preservation, dependence on position
+    differences only, and no rotation at all when every position is the same."""
+    rng = np.random.default_rng(9)
+    d, R, base = 16, 23, 10000.0
+    q = rng.standard_normal(d)
+    K = rng.standard_normal((R, d))
+    V = rng.standard_normal((R, d))
+    h = d // 2
+    theta = base ** (-2.0 * np.arange(h) / d)
+    # complex form: z_i = x_i + 1j x_{i+h}, rotated by exp(1j p theta_i); score = Re sum zq conj(zk)
+    zq = (q[:h] + 1j * q[h:]) * np.exp(1j * (R - 1) * theta)
+    zk = (K[:, :h] + 1j * K[:, h:]) * np.exp(1j * np.arange(R)[:, None] * theta)
+    lam = np.real((zk.conj() * zq).sum(axis=1)) / math.sqrt(d)
+    e = np.exp(lam - lam.max())
+    o_ref = (e / e.sum()) @ V
+    o, lse = orc.decode_attention_rope(q, K, V, base)
+    assert np.allclose(o, o_ref, rtol=1e-12, atol=1e-12)
+    assert abs(lse - (lam.max() + math.log(e.sum()))) < 1e-12
+    assert np.allclose(np.linalg.norm(orc.rope_rotate(K, np.arange(R), base), axis=1), np.linalg.norm(K, axis=1))
+    o_shift, _ = orc.decode_attention_rope(q, K, V, base, q_pos=R - 1 + 37, k_pos=np.arange(R) + 37)
+    assert np.allclose(o_shift, o, rtol=1e-9, atol=1e-11)
+    o_same, l_same = orc.decode_attention_rope(q, K, V, base, q_pos=5, k_pos=np.full(R, 5))
+    o_plain, l_plain = orc.decode_attention(q, K, V)
+    assert np.allclose(o_same, o_plain, rtol=1e-10, atol=1e-12) and abs(l_same - l_plain) < 1e-10

@@ -18,7 +18,12 @@ Parity unpinned (the paper gives no value that separates the alternatives):
   * the order in which separators leave a full Separator Cache (taken: oldest
     first), and
   * whether a streaming step attends before or after compaction (taken:
-    append, compact if full, then attend).
+    append, compact if full, then attend), and
+  * the rotary formula behind "positions within the cache" (Section 3.3 names
+    none; taken: rotate-half pairs (i, i + d/2), theta_i = base^(-2i/d), cache
+    entry r at position r, query at the last position).  rope_rotate itself is
+    pinned to the mathematics (complex-multiplication form, shift invariance,
+    norm preservation).
 """
 from __future__ import annotations
 

@@ -265,7 +265,7 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-constexpr int kDecStages = 3;
+constexpr int kDecStages = 2;
 constexpr int kDecTile = 16;  // cache rows per warp tile
 
 template <int D>
@@ -276,7 +276,7 @@ constexpr int decode_smem_bytes() {
 
 // grid (splits, Hkv, B), 4 warps.  HBM-bound: the kernel exists to stream every retained K/V row
 // once.  Each warp is an independent flash-decoding worker over its share of the split's rows:
-// 16-row K and V tiles arrive through a 3-stage cp.async ring (virtual entry -> slot mapping done
+// 16-row K and V tiles arrive through a 2-stage cp.async ring (64 KB per CTA, three CTAs per SM) (virtual entry -> slot mapping done
 // per row; rows past the end are zero-filled), the G query heads of the kv head sit in the M
 // dimension of warp-level MMAs (rows G..15 are zero), scores go through an online softmax with a
 // lazily moved reference, and O accumulates in registers.  The four warps' partials are merged
@@ -384,6 +384,7 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
       // chunks of a pair group are chunk c (elements 8c..8c+7) and chunk c + CH/2
       uint8_t* tK = wbase + (i % kDecStages) * 2 * TILEB;
       const int vrow0 = v0 + (wid + i * NW) * kDecTile;
+#pragma unroll
       for (int item = lane; item < kDecTile * (CH / 2); item += 32) {
         const int r = item / (CH / 2), c = item % (CH / 2);
         uint4* plo = reinterpret_cast<uint4*>(tK + r * ROWB + ((c ^ (r & 7)) << 4));

@@ -182,6 +182,14 @@ class Workload:
         assert self.api.sepllm_last_device_status(self.ws) == 0
         total = idx["tile_meta"][:, :, 6].astype(np.int64).sum()
         side = idx["lim"].astype(np.int64).sum()
+        # iterations of the key-stationary side pass per query head: every side tile meets the
+        # query tiles from the first one that keeps its first entry to the last
+        T, n = idx["header"].n_tiles, self.cfg["n_neighbor"]
+        self.side_iters = 0
+        for b in range(self.cfg["B"]):
+            ns = int(min(idx["n_side"][b], idx["side_pos"].shape[1]))
+            first = (idx["side_pos"][b, 0:ns:128].astype(np.int64) + n) // 128
+            self.side_iters += int(np.maximum(T - first, 0).sum())
         return int(total), int(side)
 
 
@@ -454,6 +462,7 @@ def main():
 
     # per-kernel durations and the roofline of the dominant kernel (rank 0's replica)
     kt = kernel_times(wl, min(args.steps, 10))
+    # (wl.side_iters was set by kept_pairs above)
     win_pairs = pairs - side_pairs
     kflops = {
         "attn_fwd_kernel": 4.0 * d * pairs * Hq,
@@ -465,10 +474,18 @@ def main():
     out["kernels"] = {k: {"ms": v * 1e3, "share": v / tot,
                           **({"tflops": kflops[k] / v / 1e12} if k in kflops and v > 0 else {})}
                       for k, v in kt.items()}
+    side_iters = wl.side_iters
     dom = max(kflops, key=lambda k: kt[k])
     ach = kflops[dom] / kt[dom] / 1e12
+    # DRAM bytes of the dominant kernel: one ncu capture of the 16k-token copy of this workload
+    # (profiles/ncu_full_attention_kernels_llama8b_L16k.md: 811.0 MB read + 34.4 MB written over
+    # 836 side-pass iterations per query head), scaled by iterations, which is what its Q / dO
+    # stream grows with.  Valid for bwd_dkv_kernel<side> as captured; None for anything else.
+    traffic = None
+    if dom == "bwd_dkv_kernel<side>" and cfg["d"] == 128 and cfg["Hq"] == 32 and cfg["B"] == 1:
+        traffic = (811.03e6 + 34.45e6) * side_iters / 836.0
     out["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                       "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                       "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
                        "peak_kind": f"bf16 sustained, {peaks['source']}",
                        "flops_per_launch": kflops[dom]}
 

@@ -12,7 +12,9 @@ and total capacities.
 Pins (see tests/test_oracle_*.py): brute-force loops on tiny inputs, the
 dense-causal / sliding-window special cases, row sums, finite differences,
 the closed forms of Eq. 3 and Eq. 4 with the runtime-KV values the paper
-prints, and the attention-map ratio of Table 3.
+prints, the attention-map ratio of Table 3, and for the cache a prompt leaves
+behind the description of its content that does not run the state machine
+(newest separators before a contiguous neighbour run).
 
 Parity unpinned (the paper gives no value that separates the alternatives):
   * the order in which separators leave a full Separator Cache (taken: oldest
@@ -397,6 +399,18 @@ class StreamingCache:
     def retained(self) -> List[int]:
         """Positions whose K/V the next decode step attends to."""
         return self.init + self.sep + self.window
+
+
+def cache_after_prompt(flags: Sequence[bool], a: int, s: int, w: int, c: int) -> StreamingCache:
+    """The cache a prompt leaves behind for generation (Section 3.2 "Generation",
+    Section 3.3): the state the machine above reaches after taking in the
+    prompt's tokens one by one.  The paper describes no other way of going from
+    a pre-filled prompt to the four blocks, so this is the definition the
+    hand-off from pre-filling is held to."""
+    cache = StreamingCache(a, s, w, c)
+    for fl in flags:
+        cache.update(bool(fl))
+    return cache
 
 
 def avg_neighbour_limit(w: int, c: int, a: int, s: int) -> float:

@@ -248,6 +248,42 @@ def test_streaming_cache_fifo_and_order():
     assert cache.window == [12, 13]
 
 
+def test_cache_after_prompt_has_the_content_the_blocks_are_defined_by():
+    """Without running the state machine: the neighbour run is a contiguous
+    stretch of positions ending at the prompt's last token, at least w and at
+    most c - a - Size_sep - 1 long; the Separator Cache is the newest (at most
+    s) separators between the initial tokens and that run.  Where the run
+    starts (when the compactions happened) is pinned by the hand-worked stream
+    at the end."""
+    g = np.random.default_rng(12)
+    for a, s, w, c in [(1, 2, 2, 8), (3, 4, 5, 20), (0, 3, 2, 9), (2, 0, 4, 11), (4, 16, 8, 40)]:
+        for T in [0, 1, a, a + 1, c - 1, c, c + 1, 3 * c + 2, 11 * c + 5]:
+            f = g.random(T) < 0.35
+            cache = orc.cache_after_prompt(f, a, s, w, c)
+            assert cache.init == list(range(min(T, a))) and cache.next_pos == T
+            if T <= a:
+                assert cache.sep == [] and cache.window == []
+                continue
+            lo = cache.window[0]
+            assert cache.window == list(range(lo, T))
+            seps = [j for j in range(a, lo) if f[j]]
+            assert cache.sep == seps[max(0, len(seps) - s):]
+            assert cache.window_is_sep == [bool(x) for x in f[lo:]]
+            assert cache.size_run < c
+            if cache.compactions == 0:
+                assert lo == a and T < c
+            else:
+                assert w <= len(cache.window) <= c - a - cache.size_sep - 1
+    # the worked example of the test above, cut at three prompt lengths
+    flags = [0, 1, 1, 0, 1, 1, 1, 1, 0, 0, 1, 0, 0, 0]
+    c7 = orc.cache_after_prompt(flags[:7], 1, 2, 2, 8)
+    assert (c7.init, c7.sep, c7.window, c7.compactions) == ([0], [], [1, 2, 3, 4, 5, 6], 0)
+    c8 = orc.cache_after_prompt(flags[:8], 1, 2, 2, 8)
+    assert (c8.init, c8.sep, c8.window, c8.compactions) == ([0], [4, 5], [6, 7], 1)
+    c12 = orc.cache_after_prompt(flags[:12], 1, 2, 2, 8)
+    assert (c12.init, c12.sep, c12.window, c12.compactions) == ([0], [6, 7], [9, 10, 11], 2)
+
+
 # ---------------------------------------------------------------- decode
 def test_decode_equals_last_prefill_row():
     L, d, a, n = 70, 8, 2, 9

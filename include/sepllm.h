@@ -224,6 +224,29 @@ sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, vo
                                   int32_t n_sep, const void* k_new, const void* v_new,
                                   void* stream);
 
+/* Hand-off from pre-filling to generation (Section 3.2: after the prompt only
+ * the K/V of initial, separator and neighbouring tokens are kept; Section 3.3
+ * for the four blocks).  Fills the cache with what the first prompt_len[b]
+ * tokens of sequence b leave behind: the same sizes, retained positions (in the
+ * same order), separator flags, compaction count and K/V rows as giving those
+ * tokens one by one to sepllm_cache_update on an empty cache, with both rings
+ * starting at their first slot.  The separator flag of an Initial Cache slot,
+ * which no call reads, is written as 0.  sepllm_cache_update and the decode
+ * calls continue from the result.
+ *   idesc, index   the index built from the prompts' token ids with
+ *                  n_init = desc->a and B = desc->B (its n_neighbor, tiles and
+ *                  side_cap play no part; only the prefix counts are read)
+ *   prompt_len     dev int32 [B], 0 <= prompt_len[b] <= L; NULL = L for all
+ *   K, V           dev bf16 [B][Hkv][L][d], the prompt's keys and values
+ *   state, Kc, Vc  as for sepllm_cache_update; written in full / in every
+ *                  retained slot (no sepllm_cache_init needed before)
+ * A prompt_len outside [0, L], or an index that was not built for idesc, leaves
+ * that sequence's cache empty and SEPLLM_INVALID_ARG in the device status. */
+sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
+                                       const sepllm_index_desc* idesc, const void* index,
+                                       const int32_t* prompt_len, const void* K, const void* V,
+                                       void* state, void* Kc, void* Vc, void* stream);
+
 sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* desc, size_t* bytes);
 
 /* One query per sequence over every retained entry (Section 3.2 "Generation",

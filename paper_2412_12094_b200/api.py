@@ -65,6 +65,7 @@ EXPORTS = [
     "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_static",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
+    "sepllm_cache_from_prompt",
     "sepllm_decode_workspace_bytes", "sepllm_decode", "sepllm_rope_table_bytes",
     "sepllm_rope_table_build", "sepllm_decode_rope", "sepllm_last_device_status",
     "sepllm_status_string",
@@ -202,6 +203,12 @@ def sepllm_cache_update(desc, state, Kc, Vc, new_token_ids, sep_ids, k_new, v_ne
     _check(lib().sepllm_cache_update(C.byref(desc), _ptr(state), _ptr(Kc), _ptr(Vc),
                                      _ptr(new_token_ids), p, C.c_int32(n), _ptr(k_new), _ptr(v_new),
                                      _stream()), "sepllm_cache_update")
+
+
+def sepllm_cache_from_prompt(desc, idesc, index, prompt_len, K, V, state, Kc, Vc):
+    _check(lib().sepllm_cache_from_prompt(C.byref(desc), C.byref(idesc), _ptr(index), _ptr(prompt_len),
+                                          _ptr(K), _ptr(V), _ptr(state), _ptr(Kc), _ptr(Vc), _stream()),
+           "sepllm_cache_from_prompt")
 
 
 def sepllm_decode_workspace_bytes(desc):

@@ -7,7 +7,7 @@
 //                 the Local Window Cache, the older ones the Past Window Cache
 // Decode walks "virtual" entries 0..Size_run-1 = initial, separator (oldest first), neighbour
 // (oldest first) and maps each to its slot, so only retained rows are read.
-#include "common.cuh"
+#include "attn_common.cuh"
 
 namespace sepllm {
 
@@ -213,6 +213,154 @@ cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* 
     nq.compactions = q.compactions + 1;
   }
   if (tid == 0) v.seq[b] = nq;
+}
+
+// ---------------------------------------------------------------------------
+// Prompt hand-off: the cache a pre-filled prompt leaves for generation
+// ---------------------------------------------------------------------------
+// Taking a prompt in token by token leaves (i) the first a positions in the Initial Cache, (ii) a
+// neighbour run that is the contiguous stretch [lo, T) of positions, and (iii) in the Separator
+// Cache the newest (at most s) separators of [a, lo): every compaction appends the separators it
+// passes in position order and keeps the newest s, and a tail of a tail is a tail.  Only lo needs
+// the history: a compaction happens when a + Size_sep + (t - lo) reaches c, and it moves lo to
+// t - w.  The separator counts this needs are differences of the index's prefix count `cnt`.
+constexpr int kPlanThreads = 256;
+
+struct PromptPlan {
+  int size_init, size_sep, size_win, lo, compactions;
+};
+
+// grid B.  Writes the sequence record and the per-slot position / separator flag of one sequence;
+// block 0 also writes the header.  Rings start at 0.
+__global__ void __launch_bounds__(kPlanThreads)
+prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* __restrict__ index,
+            sepllm_index_header ih, const int32_t* __restrict__ prompt_len) {
+  __shared__ PromptPlan s_plan;
+  __shared__ int s_bad;
+  const sepllm_cache_desc d = h.desc;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int L = ih.desc.L;
+  CacheView v = cache_view(state, h);
+  const int32_t* cnt = reinterpret_cast<const int32_t*>(index + ih.off_cnt) + size_t(b) * (L + 1);
+  if (tid == 0) {
+    const sepllm_index_header* dev = reinterpret_cast<const sepllm_index_header*>(index);
+    bool bad = dev->magic != SEPLLM_INDEX_MAGIC || dev->desc.B != ih.desc.B ||
+               dev->desc.L != ih.desc.L || dev->desc.n_init != ih.desc.n_init;
+    int T = L;
+    if (prompt_len) {
+      T = prompt_len[b];
+      if (T < 0 || T > L) { bad = true; T = max(0, min(T, L)); }
+    }
+    if (bad) T = 0;
+    PromptPlan p;
+    p.size_init = min(T, d.a);
+    p.size_sep = 0;
+    p.lo = d.a;
+    p.compactions = 0;
+    if (T > d.a) {
+      const int period = d.c - d.a - d.s - d.w;
+      for (;;) {
+        const int64_t t_full = int64_t(d.c) - d.a - p.size_sep + p.lo;  // tokens seen when Size_run = c
+        if (t_full > T) break;
+        const int nlo = int(t_full) - d.w;
+        if (d.s > 0) p.size_sep = min(d.s, p.size_sep + (cnt[nlo] - cnt[p.lo]));
+        p.lo = nlo;
+        ++p.compactions;
+        if (p.size_sep == d.s) {  // full for good: the remaining compactions are `period` apart
+          const int k = int((T - t_full) / period);
+          p.lo += k * period;
+          p.compactions += k;
+          break;
+        }
+      }
+    }
+    p.size_win = max(0, T - p.lo);
+    s_plan = p;
+    s_bad = bad;
+    sepllm_cache_seq q{};
+    q.size_init = p.size_init;
+    q.size_sep = p.size_sep;
+    q.size_win = p.size_win;
+    q.compactions = p.compactions;
+    q.next_pos = T;
+    v.seq[b] = q;
+    if (bad) atomicExch(&v.hdr->status, SEPLLM_INVALID_ARG);
+  }
+  if (b == 0) {
+    // header: everything but the status word, which a failing block may be writing
+    const int32_t* src = reinterpret_cast<const int32_t*>(&h);
+    int32_t* dst = reinterpret_cast<int32_t*>(v.hdr);
+    for (int k = 1 + tid; k < int(sizeof(h) / 4); k += kPlanThreads) dst[k] = src[k];
+  }
+  __syncthreads();
+  const PromptPlan p = s_plan;
+  int64_t* pos_b = v.slot_pos + size_t(b) * h.slots;
+  uint8_t* sep_b = v.slot_is_sep + size_t(b) * h.slots;
+  const int first_rank = p.size_sep > 0 ? cnt[p.lo] - p.size_sep : 0;  // among the index's side members
+  for (int slot = tid; slot < h.slots; slot += kPlanThreads) {
+    int64_t pos = 0;
+    int flag = 0;
+    if (slot < d.a) {
+      if (slot < p.size_init) pos = slot;
+    } else if (slot < d.a + d.s) {
+      const int k = slot - d.a;
+      if (k < p.size_sep) {
+        // the side member of rank r sits at the smallest j with cnt[j + 1] > r
+        const int r = first_rank + k;
+        int lo = d.a, hi = p.lo - 1;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (cnt[mid + 1] > r) hi = mid; else lo = mid + 1;
+        }
+        pos = lo;
+        flag = 1;
+      }
+    } else {
+      const int k = slot - d.a - d.s;
+      if (k < p.size_win) {
+        pos = p.lo + k;
+        flag = cnt[p.lo + k + 1] - cnt[p.lo + k];
+      }
+    }
+    pos_b[slot] = pos;
+    sep_b[slot] = uint8_t(flag);
+  }
+}
+
+constexpr int kCopyThreads = 256;
+constexpr int kCopyRows = 64;  // slots per CTA
+
+// grid (ceil(slots / kCopyRows), Hkv, B).  Copies the K and V rows of the retained positions into
+// their slots; 2 * D/8 lanes move one slot's K row and V row in 16-byte pieces.
+template <int D>
+__global__ void __launch_bounds__(kCopyThreads)
+prompt_copy(sepllm_cache_header h, const uint8_t* __restrict__ state,
+            const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V, int L,
+            __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc) {
+  constexpr int kVec = D / 8;
+  constexpr int kRowsPerPass = kCopyThreads / (2 * kVec);
+  const sepllm_cache_desc d = h.desc;
+  const int b = blockIdx.z, hk = blockIdx.y, tid = threadIdx.x;
+  CacheView v = cache_view(const_cast<uint8_t*>(state), h);
+  const sepllm_cache_seq q = v.seq[b];
+  const int64_t* pos_b = v.slot_pos + size_t(b) * h.slots;
+  const size_t src_plane = (size_t(b) * d.Hkv + hk) * size_t(L) * kVec;
+  const size_t dst_plane = (size_t(b) * d.Hkv + hk) * size_t(h.slots) * kVec;
+  const int sub = tid / (2 * kVec), l = tid % (2 * kVec);
+  const bool is_v = l >= kVec;
+  const uint4* src = reinterpret_cast<const uint4*>(is_v ? V : K) + src_plane + (is_v ? l - kVec : l);
+  uint4* dst = reinterpret_cast<uint4*>(is_v ? Vc : Kc) + dst_plane + (is_v ? l - kVec : l);
+  const int slot0 = blockIdx.x * kCopyRows;
+#pragma unroll 4
+  for (int r = sub; r < kCopyRows; r += kRowsPerPass) {
+    const int slot = slot0 + r;
+    if (slot >= h.slots) break;
+    const bool used = slot < d.a ? slot < q.size_init
+                    : slot < d.a + d.s ? slot - d.a < q.size_sep
+                                       : slot - d.a - d.s < q.size_win;
+    if (!used) continue;
+    dst[size_t(slot) * kVec] = __ldg(src + size_t(pos_b[slot]) * kVec);
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -609,6 +757,45 @@ extern "C" sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void
       h, static_cast<uint8_t*>(state), static_cast<__nv_bfloat16*>(Kc),
       static_cast<__nv_bfloat16*>(Vc), static_cast<const __nv_bfloat16*>(k_new),
       static_cast<const __nv_bfloat16*>(v_new), new_token_ids, sep);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
+                                                  const sepllm_index_desc* idesc,
+                                                  const void* index, const int32_t* prompt_len,
+                                                  const void* K, const void* V, void* state,
+                                                  void* Kc, void* Vc, void* stream_) {
+  sepllm_cache_header h;
+  sepllm_status st = fill_cache_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  sepllm_index_header ih;
+  st = fill_index_header(idesc, &ih);
+  if (st != SEPLLM_OK) return st;
+  if (!index || !K || !V || !state || !Kc || !Vc) return SEPLLM_INVALID_ARG;
+  if (idesc->B != desc->B || idesc->n_init != desc->a) return SEPLLM_INVALID_ARG;
+  if (!aligned(index, kAlign) || !aligned(state, kAlign) || !aligned(K, 16) || !aligned(V, 16) ||
+      !aligned(Kc, 16) || !aligned(Vc, 16))
+    return SEPLLM_INVALID_ARG;
+  if (desc->B > 65535 || desc->Hkv > 65535) return SEPLLM_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // the status word starts clean; everything else is written by the plan kernel
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(state, 0, sizeof(int32_t), stream));
+  prompt_plan<<<desc->B, kPlanThreads, 0, stream>>>(h, static_cast<uint8_t*>(state),
+                                                    static_cast<const uint8_t*>(index), ih,
+                                                    prompt_len);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
+  const dim3 grid((h.slots + kCopyRows - 1) / kCopyRows, desc->Hkv, desc->B);
+  if (desc->d == 128)
+    prompt_copy<128><<<grid, kCopyThreads, 0, stream>>>(
+        h, static_cast<const uint8_t*>(state), static_cast<const __nv_bfloat16*>(K),
+        static_cast<const __nv_bfloat16*>(V), idesc->L, static_cast<__nv_bfloat16*>(Kc),
+        static_cast<__nv_bfloat16*>(Vc));
+  else
+    prompt_copy<64><<<grid, kCopyThreads, 0, stream>>>(
+        h, static_cast<const uint8_t*>(state), static_cast<const __nv_bfloat16*>(K),
+        static_cast<const __nv_bfloat16*>(V), idesc->L, static_cast<__nv_bfloat16*>(Kc),
+        static_cast<__nv_bfloat16*>(Vc));
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }

@@ -4,9 +4,10 @@
 One step = the whole training-side hot path on one batch of synthetic input:
 sepllm_build_index -> sepllm_attn_fwd -> sepllm_attn_bwd.  The headline value is
 effective TFLOP/s on kept (query, key) pairs, 14*d flops per pair and query head
-(4*d forward, 10*d backward).  The streaming path (cache update + decode) and the
-index builder on a long id stream are measured in the same run and reported under
-"decode" and "index" with their own HBM rooflines.
+(4*d forward, 10*d backward).  The streaming path (cache update + decode), the
+index builder on a long id stream and the prompt hand-off into the cache are
+measured in the same run and reported under "decode", "decode_rope", "index" and
+"hand_off" with their own HBM rooflines.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
     python bench.py --impl reference ...      # the CPU oracle on a bounded sample
@@ -373,6 +374,49 @@ def bench_index_stream(device, peaks, reps=20):
                          "frac": gbs / peaks["hbm_gbs"], "traffic": None}}
 
 
+def bench_hand_off(device, peaks, reps=20, L=16384):
+    """Prompt hand-off: the streaming workload's cache filled from 16384-token prompts."""
+    from paper_2412_12094_b200 import api
+    c = inputs.DECODE_CONFIG
+    B, Hq, Hkv, d = c["B"], c["Hq"], c["Hkv"], c["d"]
+    desc = api.CacheDesc(B, Hkv, Hq, d, c["a"], c["s"], c["w"], c["c"])
+    sb, kb = api.sepllm_cache_bytes(desc)
+    state = api.alloc_bytes(sb)
+    Kc = torch.zeros(kb // 2, dtype=torch.bfloat16, device=device)
+    Vc = torch.zeros(kb // 2, dtype=torch.bfloat16, device=device)
+    ids = torch.from_numpy(inputs.decode_stream_ids(c["seed"], B, L, c["rho"])).to(device)
+    idesc = api.IndexDesc(B, L, c["a"], c["w"], len(inputs.SEP_IDS), 128, 128, L)
+    ib, scb = api.sepllm_index_bytes(idesc)
+    index, scratch = api.alloc_bytes(ib), api.alloc_bytes(scb)
+    api.sepllm_build_index(idesc, ids, inputs.SEP_IDS, index, scratch)
+    g = torch.Generator(device=device).manual_seed(c["seed"])
+    K = torch.randn((B, Hkv, L, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    V = torch.randn((B, Hkv, L, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    def call():
+        api.sepllm_cache_from_prompt(desc, idesc, index, None, K, V, state, Kc, Vc)
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    assert api.sepllm_last_device_status(state) == 0
+    sec = e0.elapsed_time(e1) / 1e3 / reps
+    st = api.read_cache_state(state)
+    rows = int((st["size_init"] + st["size_sep"] + st["size_win"]).astype(np.int64).sum())
+    algo = rows * Hkv * d * 2 * 2 * 2 + 9 * B * (c["c"] + c["s"])   # K and V rows read and written; slot metadata
+    gbs = algo / sec / 1e9
+    return {"workload": f"B32 Hkv8 d128 a4 s1024 w256 c3332 from {L}-token prompts", "us": sec * 1e6,
+            "bytes": algo, "avg_size_run": rows / B, "gpu_launches": 2 * reps,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -381,8 +425,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_long_r10", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / index-stream / e2e / CPU legs")
-    ap.add_argument("--leg", default="all", choices=["all", "decode", "decode_rope", "index"],
-                    help="decode / index: run only that secondary leg and print its JSON")
+    ap.add_argument("--leg", default="all", choices=["all", "decode", "decode_rope", "index", "hand_off"],
+                    help="run only that secondary leg and print its JSON")
     ap.add_argument("--cpu-prefix", type=int, default=8192)
     ap.add_argument("--cpu-heads", type=int, default=4)
     args = ap.parse_args()
@@ -437,6 +481,7 @@ def main():
     peaks = load_peaks()
     if args.leg != "all":
         print(json.dumps(bench_index_stream(device, peaks) if args.leg == "index"
+                         else bench_hand_off(device, peaks) if args.leg == "hand_off"
                          else bench_decode(device, peaks, rope=(args.leg == "decode_rope"))))
         return
     wl = Workload(args.workload, rank, device)
@@ -503,6 +548,7 @@ def main():
             out["decode"] = bench_decode(device, peaks)
             out["decode_rope"] = bench_decode(device, peaks, rope=True)
             out["index"] = bench_index_stream(device, peaks)
+            out["hand_off"] = bench_hand_off(device, peaks)
             if world == 1:
                 v, dt, cores, what = oracle_sample(cfg, args.cpu_heads, args.cpu_prefix)
                 out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",

@@ -155,6 +155,17 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
 sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* sep_ids, void* index, void* stream);
 
+/* Index of the fixed-interval variant (Section 4.7 "Fixed-Interval Variant",
+ * Appendix J: instead of the separators, one token every `interval` positions
+ * is attended to between the initial and the neighbouring tokens).  The side
+ * members are the first n_init positions and every position j with
+ * j % interval == 0 (the paper does not say where the intervals start; they
+ * start at position 0 here).  No token ids are read; desc->n_sep must be 0,
+ * interval >= 1.  The written index has the layout of sepllm_build_index and
+ * serves the same attention and hand-off calls.  Other arguments as there. */
+sepllm_status sepllm_build_index_fixed_interval(const sepllm_index_desc* desc, int32_t interval,
+                                                void* index, void* scratch, void* stream);
+
 /* Workspace sizes for the attention calls (bytes; either pointer may be NULL). */
 sepllm_status sepllm_attn_workspace_bytes(const sepllm_attn_desc* desc,
                                           const sepllm_index_desc* idesc, size_t* fwd_bytes,

@@ -25,7 +25,8 @@ Parity unpinned (the paper gives no value that separates the alternatives):
     none; taken: rotate-half pairs (i, i + d/2), theta_i = base^(-2i/d), cache
     entry r at position r, query at the last position).  rope_rotate itself is
     pinned to the mathematics (complex-multiplication form, shift invariance,
-    norm preservation).
+    norm preservation), and
+  * where the intervals of the fixed-interval variant start (taken: position 0).
 """
 from __future__ import annotations
 
@@ -44,6 +45,13 @@ def separator_flags(token_ids: np.ndarray, sep_ids: Iterable[int]) -> np.ndarray
     the nine separator strings; here they arrive as ids)."""
     sep = set(int(x) for x in sep_ids)
     return np.array([int(t) in sep for t in token_ids], dtype=bool)
+
+
+def fixed_interval_flags(L: int, interval: int) -> np.ndarray:
+    """Flags of the fixed-interval variant (Section 4.7, Appendix J): one token
+    every ``interval`` positions takes the separators' place.  The paper does
+    not say where the intervals start; here they start at position 0."""
+    return (np.arange(L) % int(interval)) == 0
 
 
 def mask_matrix(f: np.ndarray, a: int, n: int) -> np.ndarray:

@@ -63,6 +63,7 @@ class CacheHeader(C.Structure):
 
 EXPORTS = [
     "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_static",
+    "sepllm_build_index_fixed_interval",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
     "sepllm_cache_from_prompt",
@@ -146,6 +147,13 @@ def sepllm_build_index_static(desc: IndexDesc, token_ids: torch.Tensor, sep_ids,
     assert n == desc.n_sep
     _check(lib().sepllm_build_index_static(C.byref(desc), _ptr(token_ids), p, _ptr(index), _stream()),
            "sepllm_build_index_static")
+
+
+def sepllm_build_index_fixed_interval(desc: IndexDesc, interval: int, index: torch.Tensor,
+                                      scratch: torch.Tensor):
+    _check(lib().sepllm_build_index_fixed_interval(C.byref(desc), C.c_int32(interval), _ptr(index),
+                                                   _ptr(scratch), _stream()),
+           "sepllm_build_index_fixed_interval")
 
 
 def read_index(index: torch.Tensor) -> dict:

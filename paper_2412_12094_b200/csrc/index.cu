@@ -86,7 +86,10 @@ __device__ __forceinline__ void st_chunk_state(unsigned long long* p, uint32_t s
 constexpr int kLookbackSpins = 1 << 22;
 constexpr int kMaxTilesPerChunk = kIdxChunk / kIdxPerThread + 2;  // query tiles of >= 16 rows under one chunk
 
-// NS >= 0: compare against the first NS list entries; NS < 0: look the token up in `tab`.
+// NS >= 0: compare against the first NS list entries; NS == kSepHashed: look the token up in
+// `tab`; NS == kByPosition: no token ids, positions that are multiples of `interval` are the
+// members (the fixed-interval variant of Section 4.7 / Appendix J).
+constexpr int kSepHashed = -1, kByPosition = -2;
 template <int NS>
 __global__ void __launch_bounds__(kIdxThreads)
 index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neighbor, SepIds sep,
@@ -94,7 +97,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
            unsigned long long* __restrict__ chunk_state, int32_t* __restrict__ tickets,
            int n_chunks, int side_cap, int32_t* __restrict__ cnt, int32_t* __restrict__ lim,
            int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
-           int32_t* __restrict__ tile_meta, int T, int BM, int32_t* status) {
+           int32_t* __restrict__ tile_meta, int T, int BM, int interval, int32_t* status) {
   __shared__ int warp_buf[kIdxThreads / 32];
   __shared__ int s_chunk, s_off;
   // counts of the chunk, one pad word per 32 so that a thread's 16 consecutive words and a
@@ -103,15 +106,15 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   __shared__ int32_t tile_part[kMaxTilesPerChunk];
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  __shared__ int32_t tab_s[(NS < 0) ? kSepTableSize : 1];
+  __shared__ int32_t tab_s[(NS == kSepHashed) ? kSepTableSize : 1];
   __shared__ int lb_sum[kIdxThreads / 32], lb_found[kIdxThreads / 32];
   if (tid == 0) s_chunk = atomicAdd(&tickets[b], 1);
-  if (NS < 0) {
+  if (NS == kSepHashed) {
     for (int k = tid; k < kSepTableSize; k += kIdxThreads) tab_s[k] = tab.slot[k];
   }
   __syncthreads();
   auto is_sep = [&](int32_t tok) -> bool {
-    if (NS < 0) return tab_s[(uint32_t(tok) * tab.mult) >> (32 - kSepTableBits)] == tok;
+    if (NS == kSepHashed) return tab_s[(uint32_t(tok) * tab.mult) >> (32 - kSepTableBits)] == tok;
     return in_sep_list<(NS < 0 ? 0 : NS)>(tok, sep);
   };
   const int chunk = s_chunk;
@@ -122,7 +125,10 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   // flags of this thread's 16 consecutive positions
   const int p0 = tid * kIdxPerThread, j0 = base + p0;
   uint32_t fl = 0;
-  if (j0 + kIdxPerThread <= L && (reinterpret_cast<uintptr_t>(ids + j0) & 15) == 0) {
+  if (NS == kByPosition) {
+    for (int k = (interval - j0 % interval) % interval; k < kIdxPerThread; k += interval)
+      if (j0 + k < L) fl |= 1u << k;
+  } else if (j0 + kIdxPerThread <= L && (reinterpret_cast<uintptr_t>(ids + j0) & 15) == 0) {
     const int4* src = reinterpret_cast<const int4*>(ids + j0);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -394,7 +400,7 @@ static_assert(sizeof(sepllm_index_header) == 256, "index header is 256 bytes");
 // Launches shared by the two entry points.  `scratch` holds index_scratch_words() int32 words.
 static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_index_header& h,
                                   const int32_t* token_ids, const int32_t* sep_ids, uint8_t* blob,
-                                  int32_t* scratch, cudaStream_t stream) {
+                                  int32_t* scratch, cudaStream_t stream, int interval = 0) {
   SepIds sep;
   sep.n = desc->n_sep;
   for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k)
@@ -416,13 +422,14 @@ static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_in
       reinterpret_cast<int32_t*>(blob + h.off_lim),                                              \
       reinterpret_cast<int32_t*>(blob + h.off_side_pos),                                         \
       reinterpret_cast<int32_t*>(blob + h.off_n_side),                                           \
-      reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM,                   \
+      reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM, interval,         \
       reinterpret_cast<int32_t*>(blob))
   SepTable tab;
   tab.mult = 0;
   const bool hashed = sep.n > 0 && build_sep_table(sep_ids, sep.n, &tab);
-  if (sep.n == 0) SEPLLM_SCAN(0);
-  else if (hashed) SEPLLM_SCAN(-1);
+  if (interval > 0) SEPLLM_SCAN(kByPosition);
+  else if (sep.n == 0) SEPLLM_SCAN(0);
+  else if (hashed) SEPLLM_SCAN(kSepHashed);
   else if (sep.n <= 8) SEPLLM_SCAN(8);
   else if (sep.n <= 12) SEPLLM_SCAN(12);
   else if (sep.n <= 16) SEPLLM_SCAN(16);
@@ -459,6 +466,19 @@ extern "C" sepllm_status sepllm_build_index(const sepllm_index_desc* desc,
   if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
   return launch_index(desc, h, token_ids, sep_ids, static_cast<uint8_t*>(index),
                       static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" sepllm_status sepllm_build_index_fixed_interval(const sepllm_index_desc* desc,
+                                                           int32_t interval, void* index,
+                                                           void* scratch, void* stream_) {
+  sepllm_index_header h;
+  sepllm_status st = fill_index_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  if (interval < 1 || desc->n_sep != 0 || !index || !scratch) return SEPLLM_INVALID_ARG;
+  if (!aligned(index, kAlign) || !aligned(scratch, kAlign)) return SEPLLM_INVALID_ARG;
+  if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
+  return launch_index(desc, h, nullptr, nullptr, static_cast<uint8_t*>(index),
+                      static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream_), interval);
 }
 
 // ---------------------------------------------------------------------------

@@ -45,6 +45,24 @@ def test_mask_matches_set_construction(a, n):
     assert (orc.mask_rows(f, a, n, rows) == M[rows]).all()
 
 
+def test_fixed_interval_variant_mask():
+    """Appendix J in words: the initial tokens, one token every `interval`
+    positions, the n closest tokens.  interval = 1 keeps everything (dense
+    causal); an interval beyond the length keeps only position 0 besides the
+    initial and neighbouring tokens (the StreamingLLM pattern when a >= 1)."""
+    L, a, n = 90, 3, 7
+    for interval in (1, 2, 5, 16, 200):
+        f = orc.fixed_interval_flags(L, interval)
+        assert f.sum() == (L + interval - 1) // interval and f[0]
+        M = orc.mask_matrix(f, a, n)
+        for i in range(L):
+            kept = set(range(min(a, i + 1))) | set(range(0, i + 1, interval)) | set(range(max(0, i - n + 1), i + 1))
+            assert set(np.nonzero(M[i])[0].tolist()) == kept
+    assert (orc.mask_matrix(orc.fixed_interval_flags(L, 1), a, n) == np.tril(np.ones((L, L), bool))).all()
+    assert (orc.mask_matrix(orc.fixed_interval_flags(L, 200), a, n)
+            == orc.mask_matrix(np.zeros(L, bool), a, n)).all()
+
+
 @pytest.mark.parametrize("a,n", [(0, 1), (2, 4), (4, 16)])
 def test_forward_matches_python_loops(a, n):
     L, d = 40, 8

@@ -260,8 +260,8 @@ def kernel_times(wl: Workload, steps: int):
 
 
 def bench_decode(device, peaks, steps=4096, rope=False):
-    """Streaming workload: cache update + decode per step at the full cache shape.  rope: decode
-    with positions inside the cache (K cached un-rotated, rotated on the fly)."""
+    """Streaming workload: cache update + decode per step at the full cache shape.  rope: positions
+    inside the cache (the update keeps a rotated copy of the keys, the decode reads that)."""
     from paper_2412_12094_b200 import api
     c = inputs.DECODE_CONFIG
     B, Hq, Hkv, d = c["B"], c["Hq"], c["Hkv"], c["d"]
@@ -275,6 +275,7 @@ def bench_decode(device, peaks, steps=4096, rope=False):
     if rope:
         table = api.alloc_bytes(api.sepllm_rope_table_bytes(desc))
         api.sepllm_rope_table_build(desc, 500000.0, table)
+        Kr = torch.zeros_like(Kc)
     pool = 256
     warm = 12032                      # enough tokens to fill the separator cache (s / rho plus slack)
     T = warm + steps
@@ -285,10 +286,12 @@ def bench_decode(device, peaks, steps=4096, rope=False):
     lse = torch.empty((B, Hq), dtype=torch.float32, device=device)
 
     def step(t, ids_row):
-        api.sepllm_cache_update(desc, state, Kc, Vc, ids_row, inputs.SEP_IDS, kp[t % pool], vp[t % pool])
         if rope:
-            api.sepllm_decode_rope(desc, 0.0, qp[t % pool], state, Kc, Vc, table, o, lse, ws)
+            api.sepllm_cache_update_rope(desc, state, Kc, Vc, Kr, table, ids_row, inputs.SEP_IDS,
+                                         kp[t % pool], vp[t % pool])
+            api.sepllm_decode_rope(desc, 0.0, qp[t % pool], state, Kr, Vc, table, o, lse, ws)
         else:
+            api.sepllm_cache_update(desc, state, Kc, Vc, ids_row, inputs.SEP_IDS, kp[t % pool], vp[t % pool])
             api.sepllm_decode(desc, 0.0, qp[t % pool], state, Kc, Vc, o, lse, ws)
 
     for t in range(warm):

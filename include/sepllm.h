@@ -251,12 +251,15 @@ sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, vo
  *   K, V           dev bf16 [B][Hkv][L][d], the prompt's keys and values
  *   state, Kc, Vc  as for sepllm_cache_update; written in full / in every
  *                  retained slot (no sepllm_cache_init needed before)
+ *   Kr, rope_table NULL, or the rotated key buffer and the table of
+ *                  sepllm_cache_update_rope below: Kr is then filled as well
  * A prompt_len outside [0, L], or an index that was not built for idesc, leaves
  * that sequence's cache empty and SEPLLM_INVALID_ARG in the device status. */
 sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
                                        const sepllm_index_desc* idesc, const void* index,
                                        const int32_t* prompt_len, const void* K, const void* V,
-                                       void* state, void* Kc, void* Vc, void* stream);
+                                       void* state, void* Kc, void* Vc, void* Kr,
+                                       const void* rope_table, void* stream);
 
 sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* desc, size_t* bytes);
 
@@ -267,25 +270,41 @@ sepllm_status sepllm_decode(const sepllm_cache_desc* desc, float scale, const vo
                             const void* state, const void* Kc, const void* Vc, void* o,
                             float* lse, void* workspace, void* stream);
 
-/* Decode with positions taken inside the cache (Section 3.3, "Positional
+/* Generation with positions taken inside the cache (Section 3.3, "Positional
  * Encoding": as in StreamingLLM, the streaming setting uses an entry's place in
  * the cache, not its place in the text; Table 8 shows the effect of leaving
- * this out).  K is cached un-rotated and q is passed un-rotated; the retained
+ * this out).  Keys and queries are handed over un-rotated.  The retained
  * entries, walked as initial, separator (oldest first), neighbour (oldest
- * first), get positions 0 .. Size_run-1 and the query gets Size_run-1.  The
+ * first), have positions 0 .. Size_run-1 and the query has Size_run-1.  The
  * paper fixes no rotary formula; this library uses the rotate-half form:
  * with theta_i = base^(-2i/d), i < d/2, a vector x at position p becomes
  *   y[i]       = x[i] cos(p theta_i) - x[i + d/2] sin(p theta_i)
  *   y[i + d/2] = x[i + d/2] cos(p theta_i) + x[i] sin(p theta_i).
  * rope_table holds (cos, sin) as fp32 pairs [c][d/2]: size it with
  * sepllm_rope_table_bytes and fill it once per (desc, base) with
- * sepllm_rope_table_build (dev, 16-byte aligned).  Rotated K and q are
- * rounded to bf16 before the products.  Other arguments as sepllm_decode. */
+ * sepllm_rope_table_build (dev, 16-byte aligned).
+ *
+ * Kr is a second key buffer of Kc's size and layout (dev bf16, 16-byte
+ * aligned, caller-owned) in which every retained key stands rotated to its
+ * current position, computed in fp32 from the un-rotated key in Kc and rounded
+ * to bf16 once, however many compactions the key has been through.
+ * sepllm_cache_update_rope does what sepllm_cache_update does and keeps Kr
+ * current: an update without compaction moves no entry, so it rotates the new
+ * key only; a compaction shifts every entry behind the Initial Cache, and the
+ * call rewrites those rows of Kr from Kc.  Use it for every update of a cache
+ * that is decoded with sepllm_decode_rope (sepllm_cache_from_prompt fills Kr
+ * when given it).  sepllm_decode_rope rotates q to position Size_run-1, rounds
+ * it to bf16 and attends over Kr and Vc; other arguments as sepllm_decode. */
 sepllm_status sepllm_rope_table_bytes(const sepllm_cache_desc* desc, size_t* bytes);
 sepllm_status sepllm_rope_table_build(const sepllm_cache_desc* desc, float rope_base, void* table,
                                       void* stream);
+sepllm_status sepllm_cache_update_rope(const sepllm_cache_desc* desc, void* state, void* Kc,
+                                       void* Vc, void* Kr, const void* rope_table,
+                                       const int32_t* new_token_ids, const int32_t* sep_ids,
+                                       int32_t n_sep, const void* k_new, const void* v_new,
+                                       void* stream);
 sepllm_status sepllm_decode_rope(const sepllm_cache_desc* desc, float scale, const void* q,
-                                 const void* state, const void* Kc, const void* Vc,
+                                 const void* state, const void* Kr, const void* Vc,
                                  const void* rope_table, void* o, float* lse, void* workspace,
                                  void* stream);
 

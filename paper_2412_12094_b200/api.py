@@ -66,7 +66,7 @@ EXPORTS = [
     "sepllm_build_index_fixed_interval",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
-    "sepllm_cache_from_prompt",
+    "sepllm_cache_from_prompt", "sepllm_cache_update_rope",
     "sepllm_decode_workspace_bytes", "sepllm_decode", "sepllm_rope_table_bytes",
     "sepllm_rope_table_build", "sepllm_decode_rope", "sepllm_last_device_status",
     "sepllm_status_string",
@@ -213,9 +213,10 @@ def sepllm_cache_update(desc, state, Kc, Vc, new_token_ids, sep_ids, k_new, v_ne
                                      _stream()), "sepllm_cache_update")
 
 
-def sepllm_cache_from_prompt(desc, idesc, index, prompt_len, K, V, state, Kc, Vc):
+def sepllm_cache_from_prompt(desc, idesc, index, prompt_len, K, V, state, Kc, Vc, Kr=None, rope_table=None):
     _check(lib().sepllm_cache_from_prompt(C.byref(desc), C.byref(idesc), _ptr(index), _ptr(prompt_len),
-                                          _ptr(K), _ptr(V), _ptr(state), _ptr(Kc), _ptr(Vc), _stream()),
+                                          _ptr(K), _ptr(V), _ptr(state), _ptr(Kc), _ptr(Vc), _ptr(Kr),
+                                          _ptr(rope_table), _stream()),
            "sepllm_cache_from_prompt")
 
 
@@ -241,8 +242,15 @@ def sepllm_rope_table_build(desc, rope_base, table):
            "sepllm_rope_table_build")
 
 
-def sepllm_decode_rope(desc, scale, q, state, Kc, Vc, rope_table, o, lse, workspace):
-    _check(lib().sepllm_decode_rope(C.byref(desc), C.c_float(scale), _ptr(q), _ptr(state), _ptr(Kc),
+def sepllm_cache_update_rope(desc, state, Kc, Vc, Kr, rope_table, new_token_ids, sep_ids, k_new, v_new):
+    arr, p, n = _sep_array(sep_ids)
+    _check(lib().sepllm_cache_update_rope(C.byref(desc), _ptr(state), _ptr(Kc), _ptr(Vc), _ptr(Kr),
+                                          _ptr(rope_table), _ptr(new_token_ids), p, C.c_int32(n),
+                                          _ptr(k_new), _ptr(v_new), _stream()), "sepllm_cache_update_rope")
+
+
+def sepllm_decode_rope(desc, scale, q, state, Kr, Vc, rope_table, o, lse, workspace):
+    _check(lib().sepllm_decode_rope(C.byref(desc), C.c_float(scale), _ptr(q), _ptr(state), _ptr(Kr),
                                     _ptr(Vc), _ptr(rope_table), _ptr(o), _ptr(lse), _ptr(workspace),
                                     _stream()), "sepllm_decode_rope")
 

@@ -80,6 +80,21 @@ __device__ __forceinline__ UpdatePlan plan_update(const sepllm_cache_seq& q,
   return p;
 }
 
+// Ring starts are below the ring size and v is below the region's entry count, so one conditional
+// subtraction wraps the index (no integer division on the decode path).
+__device__ __forceinline__ int virtual_to_slot(int v, const sepllm_cache_seq& q,
+                                               const sepllm_cache_desc& d) {
+  if (v < q.size_init) return v;
+  v -= q.size_init;
+  if (v < q.size_sep) {
+    const int x = q.sep_start + v;
+    return d.a + (x >= d.s ? x - d.s : x);
+  }
+  v -= q.size_sep;
+  const int ring = d.c - d.a, x = q.win_start + v;
+  return d.a + d.s + (x >= ring ? x - ring : x);
+}
+
 constexpr int kUpdThreads = 256;
 
 // Exclusive rank of every separator among the Past Window entries, in position order.
@@ -128,11 +143,19 @@ constexpr int kMaxPast = 24576;  // int16 ranks in shared memory: 48 KB
 // The CTA that finishes last for a sequence (an arrival count in the sequence record) then
 // updates the per-slot metadata and the record, so the state changes only after every kv head
 // has planned its moves from the old one -- one launch instead of two.
+//
+// ROPE: Kr is a second key buffer with Kc's layout that holds every retained key rotated to its
+// current position inside the cache (entry v of the walk initial, separator oldest first,
+// neighbour oldest first sits at position v), computed from the un-rotated row in Kc and rounded
+// to bf16 once.  An update without a compaction moves nobody, so only the new key is rotated; a
+// compaction shifts every entry after the Initial Cache, and the CTA rewrites those rows of its
+// kv head from Kc.
+template <bool ROPE>
 __global__ void __launch_bounds__(kUpdThreads)
 cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* __restrict__ Kc,
              __nv_bfloat16* __restrict__ Vc, const __nv_bfloat16* __restrict__ k_new,
              const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ new_token_ids,
-             SepIds sep) {
+             SepIds sep, __nv_bfloat16* __restrict__ Kr, const float2* __restrict__ rope) {
   extern __shared__ int16_t flag_s[];
   __shared__ int warp_buf[32];
   __shared__ int s_last;
@@ -171,8 +194,49 @@ cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* 
     }
   }
 
+  // the sequence's record after this update (every CTA derives the same one)
+  sepllm_cache_seq nq = q;
+  nq.reserved[0] = 0;  // arrival count for the next update
+  nq.next_pos = q.next_pos + 1;
+  if (q.size_init < d.a) nq.size_init = q.size_init + 1;
+  else nq.size_win = q.size_win + 1;
+  if (p.compact) {
+    if (moves) {
+      nq.sep_start = (q.sep_start + drop) % d.s;
+      nq.size_sep = q.size_sep + m - drop;
+    }
+    nq.win_start = (q.win_start + p.n_past) % ring;
+    nq.size_win = d.w;
+    nq.compactions = q.compactions + 1;
+  }
+
+  __syncthreads();  // this CTA's append and moves are visible to all its threads
+  if (ROPE) {
+    const int size_run = nq.size_init + nq.size_sep + nq.size_win;
+    const int v_from = p.compact ? nq.size_init : size_run - 1;
+    const int half = vec / 2;  // a thread takes chunk c (elements 8c..8c+7) and its partner c + half
+    uint4* Rp = reinterpret_cast<uint4*>(Kr + plane);
+    const int items = (size_run - v_from) * half;
+    for (int item = tid; item < items; item += kUpdThreads) {
+      const int vv = v_from + item / half, c = item % half;
+      const int slot = virtual_to_slot(vv, nq, d);
+      uint4 lo = Kp[size_t(slot) * vec + c], hi = Kp[size_t(slot) * vec + c + half];
+      const float4* cs = reinterpret_cast<const float4*>(rope + size_t(vv) * (d.d / 2) + c * 8);
+      __nv_bfloat162* lo2 = reinterpret_cast<__nv_bfloat162*>(&lo);
+      __nv_bfloat162* hi2 = reinterpret_cast<__nv_bfloat162*>(&hi);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 t4 = cs[e];  // (cos, sin) of pairs 2e and 2e+1
+        const float2 x = __bfloat1622float2(lo2[e]), y = __bfloat1622float2(hi2[e]);
+        lo2[e] = __floats2bfloat162_rn(x.x * t4.x - y.x * t4.y, x.y * t4.z - y.y * t4.w);
+        hi2[e] = __floats2bfloat162_rn(y.x * t4.x + x.x * t4.y, y.y * t4.z + x.y * t4.w);
+      }
+      Rp[size_t(slot) * vec + c] = lo;
+      Rp[size_t(slot) * vec + c + half] = hi;
+    }
+  }
+
   // last kv head of the sequence to get here updates the state
-  __syncthreads();
   if (tid == 0) {
     __threadfence();
     const int prev = atomicAdd(&v.seq[b].reserved[0], 1);
@@ -188,29 +252,17 @@ cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* 
     pos_b[p.append_slot] = q.next_pos;
     sep_b[p.append_slot] = uint8_t(is_separator(new_token_ids[b], sep));
   }
-  sepllm_cache_seq nq = q;
-  nq.reserved[0] = 0;  // arrival count for the next update
-  nq.next_pos = q.next_pos + 1;
-  if (q.size_init < d.a) nq.size_init = q.size_init + 1;
-  else nq.size_win = q.size_win + 1;
-  if (p.compact) {
-    if (moves) {
-      for (int k = tid; k < p.n_past; k += kUpdThreads) {
-        const int r = flag_s[k];
-        if (r == 0) continue;
-        const int fifo = q.size_sep + (r - 1);
-        if (fifo < drop) continue;
-        const int src = wbase + (q.win_start + k) % ring;
-        const int dst = d.a + (q.sep_start + fifo) % d.s;
-        pos_b[dst] = pos_b[src];
-        sep_b[dst] = 1;
-      }
-      nq.sep_start = (q.sep_start + drop) % d.s;
-      nq.size_sep = q.size_sep + m - drop;
+  if (moves) {
+    for (int k = tid; k < p.n_past; k += kUpdThreads) {
+      const int r = flag_s[k];
+      if (r == 0) continue;
+      const int fifo = q.size_sep + (r - 1);
+      if (fifo < drop) continue;
+      const int src = wbase + (q.win_start + k) % ring;
+      const int dst = d.a + (q.sep_start + fifo) % d.s;
+      pos_b[dst] = pos_b[src];
+      sep_b[dst] = 1;
     }
-    nq.win_start = (q.win_start + p.n_past) % ring;
-    nq.size_win = d.w;
-    nq.compactions = q.compactions + 1;
   }
   if (tid == 0) v.seq[b] = nq;
 }
@@ -331,12 +383,15 @@ constexpr int kCopyThreads = 256;
 constexpr int kCopyRows = 64;  // slots per CTA
 
 // grid (ceil(slots / kCopyRows), Hkv, B).  Copies the K and V rows of the retained positions into
-// their slots; 2 * D/8 lanes move one slot's K row and V row in 16-byte pieces.
-template <int D>
+// their slots; 2 * D/8 lanes move one slot's K row and V row in 16-byte pieces.  ROPE: the K lanes
+// also write the row rotated to its position inside the cache into Kr (rings start at slot 0, so
+// the position follows from the slot).
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(kCopyThreads)
 prompt_copy(sepllm_cache_header h, const uint8_t* __restrict__ state,
             const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V, int L,
-            __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc) {
+            __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc,
+            __nv_bfloat16* __restrict__ Kr, const float2* __restrict__ rope) {
   constexpr int kVec = D / 8;
   constexpr int kRowsPerPass = kCopyThreads / (2 * kVec);
   const sepllm_cache_desc d = h.desc;
@@ -348,8 +403,10 @@ prompt_copy(sepllm_cache_header h, const uint8_t* __restrict__ state,
   const size_t dst_plane = (size_t(b) * d.Hkv + hk) * size_t(h.slots) * kVec;
   const int sub = tid / (2 * kVec), l = tid % (2 * kVec);
   const bool is_v = l >= kVec;
-  const uint4* src = reinterpret_cast<const uint4*>(is_v ? V : K) + src_plane + (is_v ? l - kVec : l);
-  uint4* dst = reinterpret_cast<uint4*>(is_v ? Vc : Kc) + dst_plane + (is_v ? l - kVec : l);
+  const int ch = is_v ? l - kVec : l;  // 16-byte chunk of the row
+  const uint4* src = reinterpret_cast<const uint4*>(is_v ? V : K) + src_plane;
+  uint4* dst = reinterpret_cast<uint4*>(is_v ? Vc : Kc) + dst_plane;
+  uint4* rdst = reinterpret_cast<uint4*>(Kr) + dst_plane;
   const int slot0 = blockIdx.x * kCopyRows;
 #pragma unroll 4
   for (int r = sub; r < kCopyRows; r += kRowsPerPass) {
@@ -359,7 +416,27 @@ prompt_copy(sepllm_cache_header h, const uint8_t* __restrict__ state,
                     : slot < d.a + d.s ? slot - d.a < q.size_sep
                                        : slot - d.a - d.s < q.size_win;
     if (!used) continue;
-    dst[size_t(slot) * kVec] = __ldg(src + size_t(pos_b[slot]) * kVec);
+    const uint4* row = src + size_t(pos_b[slot]) * kVec;
+    uint4 mine = __ldg(row + ch);
+    dst[size_t(slot) * kVec + ch] = mine;
+    if (ROPE && !is_v) {
+      // chunk ch holds elements 8ch..8ch+7; its partner in the rotation is the chunk half a row away
+      const int vpos = slot < d.a ? slot
+                     : slot < d.a + d.s ? q.size_init + (slot - d.a)
+                                        : q.size_init + q.size_sep + (slot - d.a - d.s);
+      uint4 other = __ldg(row + (ch ^ (kVec / 2)));
+      const float4* cs = reinterpret_cast<const float4*>(rope + size_t(vpos) * (D / 2) + (ch % (kVec / 2)) * 8);
+      const float sgn = (ch < kVec / 2) ? -1.f : 1.f;  // first half: x cos - y sin; second: x cos + y sin
+      __nv_bfloat162* x2 = reinterpret_cast<__nv_bfloat162*>(&mine);
+      const __nv_bfloat162* y2 = reinterpret_cast<const __nv_bfloat162*>(&other);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 t4 = cs[e];
+        const float2 x = __bfloat1622float2(x2[e]), y = __bfloat1622float2(y2[e]);
+        x2[e] = __floats2bfloat162_rn(x.x * t4.x + sgn * y.x * t4.y, x.y * t4.z + sgn * y.y * t4.w);
+      }
+      rdst[size_t(slot) * kVec + ch] = mine;
+    }
   }
 }
 
@@ -367,21 +444,6 @@ prompt_copy(sepllm_cache_header h, const uint8_t* __restrict__ state,
 // Decode: one query per sequence over the retained entries
 // ---------------------------------------------------------------------------
 constexpr int kDecThreads = 128;
-
-// Ring starts are below the ring size and v is below the region's entry count, so one conditional
-// subtraction wraps the index (no integer division on the decode path).
-__device__ __forceinline__ int virtual_to_slot(int v, const sepllm_cache_seq& q,
-                                               const sepllm_cache_desc& d) {
-  if (v < q.size_init) return v;
-  v -= q.size_init;
-  if (v < q.size_sep) {
-    const int x = q.sep_start + v;
-    return d.a + (x >= d.s ? x - d.s : x);
-  }
-  v -= q.size_sep;
-  const int ring = d.c - d.a, x = q.win_start + v;
-  return d.a + d.s + (x >= ring ? x - ring : x);
-}
 
 // ---- warp-level MMA pieces used by the decode kernel (bf16 inputs, fp32 accumulation) ----
 __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -430,10 +492,10 @@ constexpr int decode_smem_bytes() {
 // lazily moved reference, and O accumulates in registers.  The four warps' partials are merged
 // through shared memory into one (m, l, acc) record per (query head, split).
 //
-// ROPE: K rows are cached un-rotated and q arrives un-rotated; positions are indices within the
-// cache (entry v of the walk above sits at position v, the query at Size_run - 1).  Each warp
-// rotates its K tile in shared memory, pair (i, i + D/2) by the angle v * theta_i, from a table of
-// (cos, sin) per (position, i), before the MMAs read it; q is rotated while its fragments load.
+// ROPE: Kc is the rotated key buffer that the update keeps (every key already turned to its
+// position inside the cache, entry v of the walk above at position v) and q arrives un-rotated:
+// it is rotated to position Size_run - 1, pair (i, i + D/2) by the angle (Size_run - 1) * theta_i
+// from a table of (cos, sin) per (position, i), while its fragments load.
 template <int D, bool ROPE>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
@@ -527,33 +589,6 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
     cp_async_commit();
 
     const uint32_t sK = wbase_u + (i % kDecStages) * 2 * TILEB, sV = sK + TILEB;
-    if (ROPE) {
-      // rotate the tile's K rows in place: a lane takes (row, 8 pairs) items; the two 16-byte
-      // chunks of a pair group are chunk c (elements 8c..8c+7) and chunk c + CH/2
-      uint8_t* tK = wbase + (i % kDecStages) * 2 * TILEB;
-      const int vrow0 = v0 + (wid + i * NW) * kDecTile;
-#pragma unroll
-      for (int item = lane; item < kDecTile * (CH / 2); item += 32) {
-        const int r = item / (CH / 2), c = item % (CH / 2);
-        uint4* plo = reinterpret_cast<uint4*>(tK + r * ROWB + ((c ^ (r & 7)) << 4));
-        uint4* phi = reinterpret_cast<uint4*>(tK + r * ROWB + (((c + CH / 2) ^ (r & 7)) << 4));
-        uint4 lo = *plo, hi = *phi;
-        const float4* cs = reinterpret_cast<const float4*>(
-            rope + size_t(min(vrow0 + r, size_run - 1)) * (D / 2) + c * 8);
-        __nv_bfloat162* lo2 = reinterpret_cast<__nv_bfloat162*>(&lo);
-        __nv_bfloat162* hi2 = reinterpret_cast<__nv_bfloat162*>(&hi);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float4 t4 = cs[e];  // (cos, sin) of pairs 2e and 2e+1
-          const float2 x = __bfloat1622float2(lo2[e]), y = __bfloat1622float2(hi2[e]);
-          lo2[e] = __floats2bfloat162_rn(x.x * t4.x - y.x * t4.y, x.y * t4.z - y.y * t4.w);
-          hi2[e] = __floats2bfloat162_rn(y.x * t4.x + x.x * t4.y, y.y * t4.z + x.y * t4.w);
-        }
-        *plo = lo;
-        *phi = hi;
-      }
-      __syncwarp();
-    }
     // S[16 heads x 16 rows] = Q K^T
     float sc[2][4];
 #pragma unroll
@@ -729,15 +764,16 @@ extern "C" sepllm_status sepllm_cache_init(const sepllm_cache_desc* desc, void* 
   return SEPLLM_OK;
 }
 
-extern "C" sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, void* Kc,
-                                             void* Vc, const int32_t* new_token_ids,
-                                             const int32_t* sep_ids, int32_t n_sep,
-                                             const void* k_new, const void* v_new,
-                                             void* stream_) {
+static sepllm_status update_impl(const sepllm_cache_desc* desc, void* state, void* Kc, void* Vc,
+                                 const int32_t* new_token_ids, const int32_t* sep_ids,
+                                 int32_t n_sep, const void* k_new, const void* v_new, void* Kr,
+                                 const void* rope_table, bool with_rope, void* stream_) {
   sepllm_cache_header h;
   sepllm_status st = fill_cache_header(desc, &h);
   if (st != SEPLLM_OK) return st;
   if (!state || !Kc || !Vc || !new_token_ids || !k_new || !v_new) return SEPLLM_INVALID_ARG;
+  if (with_rope && (!Kr || !rope_table || !aligned(Kr, 16) || !aligned(rope_table, 16)))
+    return SEPLLM_INVALID_ARG;
   if (n_sep < 0 || (n_sep > 0 && !sep_ids)) return SEPLLM_INVALID_ARG;
   if (n_sep > SEPLLM_MAX_SEP_IDS) return SEPLLM_UNSUPPORTED;
   if (!aligned(state, kAlign) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(k_new, 16) ||
@@ -750,22 +786,45 @@ extern "C" sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void
   sep.n = n_sep;
   for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k) sep.id[k] = (k < n_sep) ? sep_ids[k] : -1;
   const size_t smem = size_t(max_past) * sizeof(int16_t);
+  auto kernel = with_rope ? cache_update<true> : cache_update<false>;
   if (smem > 40 * 1024)
-    SEPLLM_CUDA_TRY(cudaFuncSetAttribute(cache_update, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SEPLLM_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          int(smem)));
-  cache_update<<<dim3(desc->B, desc->Hkv), kUpdThreads, smem, stream>>>(
+  kernel<<<dim3(desc->B, desc->Hkv), kUpdThreads, smem, stream>>>(
       h, static_cast<uint8_t*>(state), static_cast<__nv_bfloat16*>(Kc),
       static_cast<__nv_bfloat16*>(Vc), static_cast<const __nv_bfloat16*>(k_new),
-      static_cast<const __nv_bfloat16*>(v_new), new_token_ids, sep);
+      static_cast<const __nv_bfloat16*>(v_new), new_token_ids, sep,
+      static_cast<__nv_bfloat16*>(Kr), static_cast<const float2*>(rope_table));
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
+}
+
+extern "C" sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, void* Kc,
+                                             void* Vc, const int32_t* new_token_ids,
+                                             const int32_t* sep_ids, int32_t n_sep,
+                                             const void* k_new, const void* v_new,
+                                             void* stream_) {
+  return update_impl(desc, state, Kc, Vc, new_token_ids, sep_ids, n_sep, k_new, v_new, nullptr,
+                     nullptr, false, stream_);
+}
+
+extern "C" sepllm_status sepllm_cache_update_rope(const sepllm_cache_desc* desc, void* state,
+                                                  void* Kc, void* Vc, void* Kr,
+                                                  const void* rope_table,
+                                                  const int32_t* new_token_ids,
+                                                  const int32_t* sep_ids, int32_t n_sep,
+                                                  const void* k_new, const void* v_new,
+                                                  void* stream_) {
+  return update_impl(desc, state, Kc, Vc, new_token_ids, sep_ids, n_sep, k_new, v_new, Kr,
+                     rope_table, true, stream_);
 }
 
 extern "C" sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
                                                   const sepllm_index_desc* idesc,
                                                   const void* index, const int32_t* prompt_len,
                                                   const void* K, const void* V, void* state,
-                                                  void* Kc, void* Vc, void* stream_) {
+                                                  void* Kc, void* Vc, void* Kr,
+                                                  const void* rope_table, void* stream_) {
   sepllm_cache_header h;
   sepllm_status st = fill_cache_header(desc, &h);
   if (st != SEPLLM_OK) return st;
@@ -777,6 +836,8 @@ extern "C" sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
   if (!aligned(index, kAlign) || !aligned(state, kAlign) || !aligned(K, 16) || !aligned(V, 16) ||
       !aligned(Kc, 16) || !aligned(Vc, 16))
     return SEPLLM_INVALID_ARG;
+  if ((Kr == nullptr) != (rope_table == nullptr)) return SEPLLM_INVALID_ARG;
+  if (Kr && (!aligned(Kr, 16) || !aligned(rope_table, 16))) return SEPLLM_INVALID_ARG;
   if (desc->B > 65535 || desc->Hkv > 65535) return SEPLLM_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   // the status word starts clean; everything else is written by the plan kernel
@@ -786,16 +847,15 @@ extern "C" sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
                                                     prompt_len);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   const dim3 grid((h.slots + kCopyRows - 1) / kCopyRows, desc->Hkv, desc->B);
-  if (desc->d == 128)
-    prompt_copy<128><<<grid, kCopyThreads, 0, stream>>>(
-        h, static_cast<const uint8_t*>(state), static_cast<const __nv_bfloat16*>(K),
-        static_cast<const __nv_bfloat16*>(V), idesc->L, static_cast<__nv_bfloat16*>(Kc),
-        static_cast<__nv_bfloat16*>(Vc));
-  else
-    prompt_copy<64><<<grid, kCopyThreads, 0, stream>>>(
-        h, static_cast<const uint8_t*>(state), static_cast<const __nv_bfloat16*>(K),
-        static_cast<const __nv_bfloat16*>(V), idesc->L, static_cast<__nv_bfloat16*>(Kc),
-        static_cast<__nv_bfloat16*>(Vc));
+#define SEPLLM_COPY(D, R)                                                                       \
+  prompt_copy<D, R><<<grid, kCopyThreads, 0, stream>>>(                                         \
+      h, static_cast<const uint8_t*>(state), static_cast<const __nv_bfloat16*>(K),              \
+      static_cast<const __nv_bfloat16*>(V), idesc->L, static_cast<__nv_bfloat16*>(Kc),          \
+      static_cast<__nv_bfloat16*>(Vc), static_cast<__nv_bfloat16*>(Kr),                         \
+      static_cast<const float2*>(rope_table))
+  if (desc->d == 128) { if (Kr) SEPLLM_COPY(128, true); else SEPLLM_COPY(128, false); }
+  else { if (Kr) SEPLLM_COPY(64, true); else SEPLLM_COPY(64, false); }
+#undef SEPLLM_COPY
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }

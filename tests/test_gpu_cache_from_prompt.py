@@ -167,3 +167,45 @@ def test_hand_off_rejects_what_it_cannot_use():
     torch.cuda.synchronize()
     assert api.sepllm_last_device_status(gc.state) == api.INVALID_ARG
     assert api.read_cache_state(gc.state)["next_pos"].tolist() == [0, 0]
+
+
+def test_hand_off_fills_the_rotated_key_buffer():
+    """Hand-off with Kr, then rotary updates: the rotary decode agrees exactly with a cache that took
+    every token through sepllm_cache_update_rope (same rotated rows, same order)."""
+    B, Hkv, Hq, d, a, s, w, c = 2, 2, 8, 128, 4, 16, 32, 100
+    L, more = 500, 130
+    ids, K, V = _prompt(95, B, Hkv, L + more, d, 0.15)
+    Kd, Vd = K.cuda(), V.cuda()
+    ids_d = torch.from_numpy(np.ascontiguousarray(ids.T)).cuda()
+    fast, slow = GpuCache(B, Hkv, Hq, d, a, s, w, c), GpuCache(B, Hkv, Hq, d, a, s, w, c)
+    table = api.alloc_bytes(api.sepllm_rope_table_bytes(fast.desc))
+    api.sepllm_rope_table_build(fast.desc, 10000.0, table)
+    Kr_f, Kr_s = torch.zeros_like(fast.Kc), torch.zeros_like(slow.Kc)
+    idesc, index = build_index(np.ascontiguousarray(ids[:, :L]), inputs.SEP_IDS, a, 64)
+    api.sepllm_cache_from_prompt(fast.desc, idesc, index, None, Kd[:, :, :L].contiguous(),
+                                 Vd[:, :, :L].contiguous(), fast.state, fast.Kc, fast.Vc, Kr_f, table)
+    q = inputs.normal_bf16(95, 33, (B, Hq, d)).cuda()
+
+    def decode(gc, Kr):
+        o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+        api.sepllm_decode_rope(gc.desc, 0.0, q, gc.state, Kr, gc.Vc, table, o, lse, gc.ws)
+        return o, lse
+
+    for t in range(L + more):
+        api.sepllm_cache_update_rope(slow.desc, slow.state, slow.Kc, slow.Vc, Kr_s, table, ids_d[t],
+                                     inputs.SEP_IDS, Kd[:, :, t].contiguous(), Vd[:, :, t].contiguous())
+        if t >= L:
+            api.sepllm_cache_update_rope(fast.desc, fast.state, fast.Kc, fast.Vc, Kr_f, table, ids_d[t],
+                                         inputs.SEP_IDS, Kd[:, :, t].contiguous(), Vd[:, :, t].contiguous())
+        if t in (L - 1, L + 40, L + more - 1):
+            (o1, l1), (o2, l2) = decode(fast, Kr_f), decode(slow, Kr_s)
+            torch.cuda.synchronize()
+            assert torch.equal(o1, o2) and torch.equal(l1, l2), t
+    sf, ss = api.read_cache_state(fast.state), api.read_cache_state(slow.state)
+    for b in range(B):
+        assert fast.regions(sf, b) == slow.regions(ss, b)
+        rows_f = Kr_f.view(B, Hkv, fast.slots, d)[b][:, fast.slot_of_virtual(sf, b)]
+        rows_s = Kr_s.view(B, Hkv, slow.slots, d)[b][:, slow.slot_of_virtual(ss, b)]
+        assert torch.equal(rows_f, rows_s)
+    assert ss["compactions"].min() >= 5

@@ -1,4 +1,5 @@
-"""sepllm_decode_rope (positions inside the cache) against the oracle's rotary decode."""
+"""sepllm_cache_update_rope / sepllm_decode_rope (positions inside the cache) against the oracle's
+rotary decode."""
 import numpy as np
 import pytest
 import torch
@@ -10,14 +11,29 @@ from tests.test_gpu_cache import GpuCache
 
 pytestmark = pytest.mark.gpu
 
-# The kernel rounds the rotated K rows and the rotated q to bf16 before the tensor-core products
+# The library rounds the rotated K rows and the rotated q to bf16 before the tensor-core products
 # (the oracle rotates in fp64), so every score carries two relative roundings of 2^-9 per term:
 # about 2^-9 * sqrt(2) * |q||k| / d ~ 3e-3 rms for N(0,1) inputs.  LSE is a weighted mean of the
 # scores' errors, hence the looser bound than for the plain decode; O keeps the common tolerance.
 TOL_LSE_ROPE = 1e-2
 
 
-def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at):
+def _check_rotated_keys(gc, Kr, st, base):
+    """Every retained row of Kr is the row of Kc turned to its position inside the cache: half a
+    bf16 ulp from the rounding plus the fp32 angle (position * theta carries 2^-24 relative error,
+    under 3e-4 rad at position 4000)."""
+    d = gc.desc
+    Kc = gc.Kc.view(d.B, d.Hkv, gc.slots, d.d).double().cpu().numpy()
+    Kr = Kr.view(d.B, d.Hkv, gc.slots, d.d).double().cpu().numpy()
+    for b in range(d.B):
+        slots = gc.slot_of_virtual(st, b)
+        for hk in range(d.Hkv):
+            ref = orc.rope_rotate(Kc[b, hk][slots], np.arange(len(slots)), base)
+            err = np.abs(Kr[b, hk][slots] - ref)
+            assert (err <= 2.0 ** -8 * np.maximum(1.0, np.abs(ref)) + 1e-3).all(), (b, hk, err.max())
+
+
+def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at, keys_every=0):
     ids = inputs.decode_stream_ids(seed, B, steps, rho)
     kp, vp, qp = inputs.decode_kv_pool(seed, steps, B, Hkv, Hq, d)
     kd, vd, qd = kp.cuda(), vp.cuda(), qp.cuda()
@@ -25,16 +41,22 @@ def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at):
     gc = GpuCache(B, Hkv, Hq, d, a, s, w, c)
     table = api.alloc_bytes(api.sepllm_rope_table_bytes(gc.desc))
     api.sepllm_rope_table_build(gc.desc, base, table)
+    Kr = torch.full_like(gc.Kc, float("nan"))      # a row the update failed to write would show
     G = Hq // Hkv
     o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device="cuda")
     lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
     for t in range(steps):
-        gc.update(ids_d[t], kd[t], vd[t])
+        api.sepllm_cache_update_rope(gc.desc, gc.state, gc.Kc, gc.Vc, Kr, table, ids_d[t], inputs.SEP_IDS,
+                                     kd[t], vd[t])
+        if keys_every and t % keys_every == 0:
+            torch.cuda.synchronize()
+            _check_rotated_keys(gc, Kr, api.read_cache_state(gc.state), base)
         if t not in check_at:
             continue
-        api.sepllm_decode_rope(gc.desc, 0.0, qd[t], gc.state, gc.Kc, gc.Vc, table, o, lse, gc.ws)
+        api.sepllm_decode_rope(gc.desc, 0.0, qd[t], gc.state, Kr, gc.Vc, table, o, lse, gc.ws)
         torch.cuda.synchronize()
         st = api.read_cache_state(gc.state)
+        _check_rotated_keys(gc, Kr, st, base)
         Kc = gc.Kc.view(B, Hkv, gc.slots, d).float().cpu().numpy()
         Vc = gc.Vc.view(B, Hkv, gc.slots, d).float().cpu().numpy()
         on, ln = o.float().cpu().numpy(), lse.cpu().numpy()
@@ -52,9 +74,35 @@ def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at):
 @pytest.mark.parametrize("d,Hq,Hkv", [(64, 2, 2), (128, 8, 2), (128, 4, 1)])
 def test_rope_decode_small(d, Hq, Hkv):
     _drive(2, Hkv, Hq, d, a=2, s=5, w=4, c=20, steps=90, rho=0.3, seed=70 + d + Hq, base=10000.0,
-           check_at={0, 1, 5, 19, 20, 21, 47, 89})
+           check_at={0, 1, 5, 19, 20, 21, 47, 89}, keys_every=1)
 
 
 def test_rope_decode_medium_llama_base():
     _drive(3, 2, 8, 128, a=4, s=64, w=256, c=800, steps=1700, rho=0.12, seed=77, base=500000.0,
            check_at={300, 799, 800, 1250, 1699})
+
+
+def test_rope_no_separator_cache_and_no_initial_tokens():
+    _drive(1, 1, 2, 64, a=3, s=0, w=5, c=12, steps=60, rho=0.5, seed=78, base=10000.0,
+           check_at={0, 11, 12, 59}, keys_every=1)
+    _drive(1, 1, 1, 64, a=0, s=3, w=2, c=9, steps=60, rho=0.5, seed=79, base=10000.0,
+           check_at={0, 8, 9, 59}, keys_every=1)
+
+
+def test_rope_state_machine_is_the_plain_one():
+    """The rotary update changes Kr only: state, Kc and Vc end up as with sepllm_cache_update."""
+    B, Hkv, Hq, d, a, s, w, c, steps = 2, 2, 4, 128, 2, 6, 4, 24, 150
+    ids = inputs.decode_stream_ids(81, B, steps, 0.3)
+    kp, vp, _ = inputs.decode_kv_pool(81, steps, B, Hkv, Hq, d)
+    kd, vd = kp.cuda(), vp.cuda()
+    ids_d = torch.from_numpy(np.ascontiguousarray(ids.T)).cuda()
+    plain, rot = GpuCache(B, Hkv, Hq, d, a, s, w, c), GpuCache(B, Hkv, Hq, d, a, s, w, c)
+    table = api.alloc_bytes(api.sepllm_rope_table_bytes(rot.desc))
+    api.sepllm_rope_table_build(rot.desc, 10000.0, table)
+    Kr = torch.zeros_like(rot.Kc)
+    for t in range(steps):
+        plain.update(ids_d[t], kd[t], vd[t])
+        api.sepllm_cache_update_rope(rot.desc, rot.state, rot.Kc, rot.Vc, Kr, table, ids_d[t],
+                                     inputs.SEP_IDS, kd[t], vd[t])
+    torch.cuda.synchronize()
+    assert torch.equal(plain.state, rot.state) and torch.equal(plain.Kc, rot.Kc) and torch.equal(plain.Vc, rot.Vc)

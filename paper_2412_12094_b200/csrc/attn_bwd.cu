@@ -335,36 +335,42 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive_warp(bar_sl);  // the S columns may be overwritten from here on
-        if (need_mask) {
+        // packed fp32 pairs: one multiply-add instruction per two scores
+        const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+        const unsigned long long nlse2 = pack_f32x2(neg_lse2, neg_lse2);
 #pragma unroll
-          for (int c = 0; c < 2; ++c)
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
+          for (int e = 0; e < 32; e += 2) {
+            const float2 a = unpack_f32x2(fma_f32x2(
+                pack_f32x2(__uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1])), scale2, nlse2));
+            float p0 = ex2(a.x), p1 = ex2(a.y);
+            if (need_mask) {
               const int col = u * 64 + c * 32 + e;
-              const float pr = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2));
-              sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? pr : 0.f);
+              p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
+              p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
             }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 2; ++c)
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, neg_lse2)));
-        }
+            sv[c][e] = __float_as_uint(p0);
+            sv[c][e + 1] = __float_as_uint(p1);
+          }
         // phase B: dS = P (dP - Delta)
         wait(bar_dp, gi & 1);
         tc_fence_after();
         uint32_t pk[32];
+        const unsigned long long ndelta2 = pack_f32x2(-delta_i, -delta_i);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t dp[32];
           tmem_ld32(tdP + c * 32, dp);
           tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; e += 2)
-            pk[c * 16 + (e >> 1)] =
-                pack_bf16(__uint_as_float(sv[c][e]) * (__uint_as_float(dp[e]) - delta_i),
-                          __uint_as_float(sv[c][e + 1]) * (__uint_as_float(dp[e + 1]) - delta_i));
+          for (int e = 0; e < 32; e += 2) {
+            const unsigned long long t2 = add_f32x2(
+                pack_f32x2(__uint_as_float(dp[e]), __uint_as_float(dp[e + 1])), ndelta2);
+            const float2 ds = unpack_f32x2(mul_f32x2(
+                pack_f32x2(__uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1])), t2));
+            pk[c * 16 + (e >> 1)] = pack_bf16(ds.x, ds.y);
+          }
         }
         // packed dS over the first half of this thread's own dP columns
         tmem_st32(tdP, pk);
@@ -614,8 +620,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const float2 v0 = (q < p.L) ? p.stats[base + q] : make_float2(INFINITY, 0.f);
         const float2 v1 = (q + 64 < p.L) ? p.stats[base + q + 64] : make_float2(INFINITY, 0.f);
         if (it >= 1) wait(bar_pds, (it - 1) & 1);
-        s_stat[i] = make_float2(-v0.x, v0.y);
-        s_stat[64 + i] = make_float2(-v1.x, v1.y);
+        // -LSE of the 128 query columns, then -Delta of the 128: the arithmetic warps read two
+        // neighbouring columns' values as one packed fp32 pair
+        float* sf = reinterpret_cast<float*>(s_stat);
+        sf[i] = -v0.x;
+        sf[64 + i] = -v1.x;
+        sf[128 + i] = -v0.y;
+        sf[192 + i] = -v1.y;
         mbar_arrive_warp(bar_sf);
       }
     }
@@ -659,28 +670,28 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive_warp(bar_sl);  // the S^T columns may be overwritten from here on
-      // two columns' (-LSE in log2 units, Delta) per shared-memory load
-      const float4* stat2 = reinterpret_cast<const float4*>(s_stat + u * 64);
+      // two columns' -LSE (log2 units) and -Delta per shared-memory load, as packed fp32 pairs
+      const unsigned long long* nlse2 =
+          reinterpret_cast<const unsigned long long*>(reinterpret_cast<const float*>(s_stat) + u * 64);
+      const unsigned long long* ndel2 = nlse2 + 64;
+      const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float2 a = unpack_f32x2(fma_f32x2(
+              pack_f32x2(__uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1])), scale2,
+              nlse2[(c * 32 + e) >> 1]));
+          sv[c][e] = __float_as_uint(ex2(a.x));
+          sv[c][e + 1] = __float_as_uint(ex2(a.y));
+        }
       if (need_mask) {
 #pragma unroll
         for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
+          for (int e = 0; e < 32; ++e) {
             const int col = u * 64 + c * 32 + e;
-            const float4 sd = stat2[(c * 32 + e) >> 1];
-            const float p0 = ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, sd.x));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, sd.z));
-            sv[c][e] = __float_as_uint((col >= c_lo && col < c_hi) ? p0 : 0.f);
-            sv[c][e + 1] = __float_as_uint((col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f);
-          }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float4 sd = stat2[(c * 32 + e) >> 1];
-            sv[c][e] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e]), p.scale_log2, sd.x)));
-            sv[c][e + 1] = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c][e + 1]), p.scale_log2, sd.z)));
+            sv[c][e] = (col >= c_lo && col < c_hi) ? sv[c][e] : 0u;
           }
       }
       // phase B: dS^T = P^T (dP^T - Delta)
@@ -694,11 +705,12 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          const float4 sd = stat2[(c * 32 + e) >> 1];
           const float p0 = __uint_as_float(sv[c][e]), p1 = __uint_as_float(sv[c][e + 1]);
           pkp[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
-          pkd[c * 16 + (e >> 1)] = pack_bf16(p0 * (__uint_as_float(dp[e]) - sd.y),
-                                             p1 * (__uint_as_float(dp[e + 1]) - sd.w));
+          const unsigned long long t2 = add_f32x2(
+              pack_f32x2(__uint_as_float(dp[e]), __uint_as_float(dp[e + 1])), ndel2[(c * 32 + e) >> 1]);
+          const float2 ds = unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1), t2));
+          pkd[c * 16 + (e >> 1)] = pack_bf16(ds.x, ds.y);
         }
       }
       tmem_st32(tdPT, pkp);

@@ -327,7 +327,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sreg[c][e]));
+            for (int e = 0; e < 32; e += 8)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mx4[k] = max3(mx4[k], __uint_as_float(sreg[c][e + k]), __uint_as_float(sreg[c][e + 4 + k]));
         }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
         // lazy rescale: move the reference only when the maximum grew by more than 2^8
@@ -339,17 +342,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           rescale = true;
         }
         const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-        float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+        const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+        const unsigned long long negm2 = pack_f32x2(neg_m, neg_m);
+        unsigned long long ps2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed partial sums (+0.0f pairs)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sreg[c][e]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(sreg[c][e + 1]), p.scale_log2, neg_m));
-            ps4[(e >> 1) & 3] += p0 + p1;
+            const float2 a = unpack_f32x2(fma_f32x2(
+                pack_f32x2(__uint_as_float(sreg[c][e]), __uint_as_float(sreg[c][e + 1])), scale2, negm2));
+            const float p0 = ex2(a.x), p1 = ex2(a.y);
+            ps2[(e >> 1) & 3] = add_f32x2(ps2[(e >> 1) & 3], pack_f32x2(p0, p1));
             sreg[c][e >> 1] = pack_bf16(p0, p1);
           }
-        l_sum = l_sum * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+        const float2 sm = unpack_f32x2(add_f32x2(add_f32x2(ps2[0], ps2[1]), add_f32x2(ps2[2], ps2[3])));
+        l_sum = l_sum * corr + (sm.x + sm.y);
 
         // S_x(j) complete means PV_x of the previous tile is complete too: O_x is quiescent
         if (n_done > 0 && __any_sync(0xffffffffu, rescale)) {

@@ -236,7 +236,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const uint32_t v_lo0 = desc_lo(smem_u32(sV), kTileBlockBytes);
       int n_pv[2] = {0, 0};  // PV MMAs issued per slot
       bool q_seen[2] = {false, false};
+      // Every barrier test, fence and commit costs this thread 50-300 cycles during which the
+      // tensor pipe drains, so each is done once per step: the K and V tiles are waited for by
+      // the first slot that needs them, and the only tcgen05 fence follows the wait for P (the
+      // other waits guard TMA data, which the barrier itself makes visible).
       for (int s = 0; s <= n_tiles; ++s) {
+        bool k_waited = false, v_waited = false;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           const SlotGeom& g = x ? g1 : g0;
@@ -244,7 +249,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           if (s >= 1 && slot_active(g, ns, wlo, s - 1)) {
             const int j = s - 1, st = j % NST;
             wait(bar_p + x, n_pv[x] & 1);
-            wait(bar_vf + st, (j / NST) & 1);
+            if (!v_waited) { wait(bar_vf + st, (j / NST) & 1); v_waited = true; }
             tc_fence_after();
             const uint32_t v_lo = v_lo0 + st * (C::kTile >> 4);
             umma_ts_lo(tO, tS, v_lo, idesc_o, n_pv[x] > 0);
@@ -256,8 +261,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           if (s < n_tiles && slot_active(g, ns, wlo, s)) {
             const int st = s % NST;
             if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
-            wait(bar_kf + st, (s / NST) & 1);
-            tc_fence_after();
+            if (!k_waited) { wait(bar_kf + st, (s / NST) & 1); k_waited = true; }
             const uint32_t k_lo = k_lo0 + st * (C::kTile >> 4);
 #pragma unroll
             for (int k = 0; k < D / 16; ++k)
@@ -311,19 +315,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           c_lo = row - p.n_neighbor + 1 - key0;
           need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
         }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        if (need_mask) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const int col = c * 32 + e;
-              float s = __uint_as_float(sreg[c][e]);
-              s = (col >= c_lo && col < c_hi) ? s : -INFINITY;
-              sreg[c][e] = __float_as_uint(s);
-              mx4[e & 3] = fmaxf(mx4[e & 3], s);
-            }
-        } else {
+        // Reference exponent.  A tile that needs no mask and finds a reference already set skips
+        // the maximum: its exponentials are taken against the old reference, which is exact as
+        // long as nothing overflows (fp32 sums and bf16 P have the range for a lag of 2^64), and
+        // the row sum tells if it did.  Otherwise the reference moves when the tile's maximum
+        // exceeds it by more than 2^8.
+        auto tile_max = [&]() -> float {
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -331,32 +329,56 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 #pragma unroll
               for (int k = 0; k < 4; ++k)
                 mx4[k] = max3(mx4[k], __uint_as_float(sreg[c][e + k]), __uint_as_float(sreg[c][e + 4 + k]));
+          return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+        };
+        // P = 2^(S * scale - m_ref) packed over sreg[c][0..15]; returns the row sum of the tile
+        auto exponentials = [&]() -> float {
+          const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+          const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+          const unsigned long long negm2 = pack_f32x2(neg_m, neg_m);
+          unsigned long long ps2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed partial sums
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float2 a = unpack_f32x2(fma_f32x2(
+                  pack_f32x2(__uint_as_float(sreg[c][e]), __uint_as_float(sreg[c][e + 1])), scale2, negm2));
+              const float p0 = ex2(a.x), p1 = ex2(a.y);
+              ps2[(e >> 1) & 3] = add_f32x2(ps2[(e >> 1) & 3], pack_f32x2(p0, p1));
+              sreg[c][e >> 1] = pack_bf16(p0, p1);
+            }
+          const float2 sm = unpack_f32x2(add_f32x2(add_f32x2(ps2[0], ps2[1]), add_f32x2(ps2[2], ps2[3])));
+          return sm.x + sm.y;
+        };
+        auto move_reference = [&](float mx, float& corr, bool& rescale) {
+          if (mx > m_ref + 8.f) {
+            corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
+            m_ref = mx;
+            rescale = true;
+          }
+        };
+        if (need_mask) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int col = c * 32 + e;
+              sreg[c][e] = (col >= c_lo && col < c_hi) ? sreg[c][e] : 0xff800000u;  // -inf
+            }
         }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
-        // lazy rescale: move the reference only when the maximum grew by more than 2^8
         float corr = 1.f;
         bool rescale = false;
-        if (mx > m_ref + 8.f) {
-          corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
-          m_ref = mx;
-          rescale = true;
+        if (need_mask || m_ref == -INFINITY) move_reference(tile_max(), corr, rescale);
+        float tile_sum = exponentials();
+        if (__any_sync(0xffffffffu, !(tile_sum < 1.8e19f))) {
+          // some row of this warp ran past the range: take the tile again with its own maximum
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, sreg[c]);
+          tmem_ld_wait();
+          move_reference(tile_max(), corr, rescale);
+          tile_sum = exponentials();
         }
-        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-        const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
-        const unsigned long long negm2 = pack_f32x2(neg_m, neg_m);
-        unsigned long long ps2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed partial sums (+0.0f pairs)
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float2 a = unpack_f32x2(fma_f32x2(
-                pack_f32x2(__uint_as_float(sreg[c][e]), __uint_as_float(sreg[c][e + 1])), scale2, negm2));
-            const float p0 = ex2(a.x), p1 = ex2(a.y);
-            ps2[(e >> 1) & 3] = add_f32x2(ps2[(e >> 1) & 3], pack_f32x2(p0, p1));
-            sreg[c][e >> 1] = pack_bf16(p0, p1);
-          }
-        const float2 sm = unpack_f32x2(add_f32x2(add_f32x2(ps2[0], ps2[1]), add_f32x2(ps2[2], ps2[3])));
-        l_sum = l_sum * corr + (sm.x + sm.y);
+        l_sum = l_sum * corr + tile_sum;
 
         // S_x(j) complete means PV_x of the previous tile is complete too: O_x is quiescent
         if (n_done > 0 && __any_sync(0xffffffffu, rescale)) {

@@ -75,3 +75,25 @@ def test_fwd_rejects_unsupported():
     with pytest.raises(api.SepllmError) as e:
         api.sepllm_attn_workspace_bytes(api.AttnDesc(1, 3, 2, 64, 256, 0.0, 0), idesc)
     assert e.value.code == api.INVALID_ARG
+
+
+def test_fwd_scores_that_outgrow_the_first_tiles_reference():
+    """Unmasked tiles after the first keep the row's old reference exponent; here the later keys
+    score 2^100 above the first tile's, which must be caught and the tile redone with its own
+    maximum (and a jump of 2^40, which must go through without that)."""
+    B, Hq, Hkv, L, d = 1, 2, 1, 640, 64
+    ids = inputs.token_ids(5, B, L, 0.0)
+    _, _, V, _ = inputs.qkv_do(321, B, Hq, Hkv, L, d)
+    for c in (3.0, 1.875):                      # sqrt(d) c^2 log2(e) = 104 and 40.6
+        Q = torch.full((B, Hq, L, d), c, dtype=torch.bfloat16)
+        K = torch.full((B, Hkv, L, d), c, dtype=torch.bfloat16)
+        K[:, :, :128] = 0                        # the first key tile scores 0
+        K[:, :, 300:] *= -1                      # and the last keys fall far below again
+        idesc, index = build_index(ids, inputs.SEP_IDS, 0, L)     # dense causal
+        O, LSE = attn_fwd(Q.cuda(), K.cuda(), V.cuda(), idesc, index)
+        Oref, LSEref = orc.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(),
+                                    flags_of(ids, inputs.SEP_IDS), 0, L)
+        assert_close(O.float().cpu().numpy(), Oref, TOL_O, f"O c={c}")
+        # LSE reaches 72 here: the fp32 product score * (scale * log2 e) carries 2^-24 of that per
+        # rounding, so the bound scales with the magnitude beyond the workloads' |LSE| < 8
+        assert np.abs(LSE.cpu().numpy() - LSEref).max() <= TOL_LSE * max(1.0, np.abs(LSEref).max() / 8)

@@ -245,8 +245,10 @@ sepllm_status sepllm_cache_update(const sepllm_cache_desc* desc, void* state, vo
  * which no call reads, is written as 0.  sepllm_cache_update and the decode
  * calls continue from the result.
  *   idesc, index   the index built from the prompts' token ids with
- *                  n_init = desc->a and B = desc->B (its n_neighbor, tiles and
- *                  side_cap play no part; only the prefix counts are read)
+ *                  n_init = desc->a and B = desc->B (its n_neighbor and tiles
+ *                  play no part; the prefix counts and the side list are read,
+ *                  and a side list cut short by side_cap is made up for from
+ *                  the counts)
  *   prompt_len     dev int32 [B], 0 <= prompt_len[b] <= L; NULL = L for all
  *   K, V           dev bf16 [B][Hkv][L][d], the prompt's keys and values
  *   state, Kc, Vc  as for sepllm_cache_update; written in full / in every

@@ -276,7 +276,7 @@ cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* 
 // passes in position order and keeps the newest s, and a tail of a tail is a tail.  Only lo needs
 // the history: a compaction happens when a + Size_sep + (t - lo) reaches c, and it moves lo to
 // t - w.  The separator counts this needs are differences of the index's prefix count `cnt`.
-constexpr int kPlanThreads = 256;
+constexpr int kPlanThreads = 1024;
 
 struct PromptPlan {
   int size_init, size_sep, size_win, lo, compactions;
@@ -294,10 +294,13 @@ prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* _
   const int L = ih.desc.L;
   CacheView v = cache_view(state, h);
   const int32_t* cnt = reinterpret_cast<const int32_t*>(index + ih.off_cnt) + size_t(b) * (L + 1);
+  const int32_t* side_pos =
+      reinterpret_cast<const int32_t*>(index + ih.off_side_pos) + size_t(b) * ih.desc.side_cap;
   if (tid == 0) {
     const sepllm_index_header* dev = reinterpret_cast<const sepllm_index_header*>(index);
     bool bad = dev->magic != SEPLLM_INDEX_MAGIC || dev->desc.B != ih.desc.B ||
-               dev->desc.L != ih.desc.L || dev->desc.n_init != ih.desc.n_init;
+               dev->desc.L != ih.desc.L || dev->desc.n_init != ih.desc.n_init ||
+               dev->desc.side_cap != ih.desc.side_cap;
     int T = L;
     if (prompt_len) {
       T = prompt_len[b];
@@ -357,14 +360,19 @@ prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* _
     } else if (slot < d.a + d.s) {
       const int k = slot - d.a;
       if (k < p.size_sep) {
-        // the side member of rank r sits at the smallest j with cnt[j + 1] > r
+        // the side member of rank r: the index's side list has it unless the list was cut short,
+        // then it is the smallest j with cnt[j + 1] > r
         const int r = first_rank + k;
-        int lo = d.a, hi = p.lo - 1;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (cnt[mid + 1] > r) hi = mid; else lo = mid + 1;
+        if (r < ih.desc.side_cap) {
+          pos = side_pos[r];
+        } else {
+          int lo = d.a, hi = p.lo - 1;
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (cnt[mid + 1] > r) hi = mid; else lo = mid + 1;
+          }
+          pos = lo;
         }
-        pos = lo;
         flag = 1;
       }
     } else {

@@ -209,3 +209,21 @@ def test_hand_off_fills_the_rotated_key_buffer():
         rows_s = Kr_s.view(B, Hkv, slow.slots, d)[b][:, slow.slot_of_virtual(ss, b)]
         assert torch.equal(rows_f, rows_s)
     assert ss["compactions"].min() >= 5
+
+
+def test_hand_off_with_a_side_list_cut_short():
+    """side_cap below the number of side members: the index reports it, its prefix counts are still
+    complete, and the hand-off finds the separators the list lacks from the counts."""
+    B, Hkv, Hq, d, a, s, w, c = 2, 1, 2, 64, 2, 12, 4, 40
+    L = 600
+    ids, K, V = _prompt(97, B, Hkv, L, d, 0.3)
+    f = np.isin(ids, inputs.SEP_IDS)
+    gc = GpuCache(B, Hkv, Hq, d, a, s, w, c)
+    idesc, index = build_index(ids, inputs.SEP_IDS, a, 16, side_cap=20)
+    api.sepllm_cache_from_prompt(gc.desc, idesc, index, None, K.cuda(), V.cuda(), gc.state, gc.Kc, gc.Vc)
+    torch.cuda.synchronize()
+    assert api.sepllm_last_device_status(index) == api.CAPACITY_EXCEEDED
+    assert api.sepllm_last_device_status(gc.state) == 0
+    oc = [orc.cache_after_prompt(f[b], a, s, w, c) for b in range(B)]
+    _check_against_oracle(gc, oc, f, K, V)
+    assert all(len(x.sep) == s for x in oc)

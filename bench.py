@@ -154,7 +154,7 @@ class Workload:
         self.dK = torch.empty_like(self.K)
         self.dV = torch.empty_like(self.V)
         self.out_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (self.O, self.dQ, self.dK, self.dV)]
-        self.launches_per_step = 2 + 2 + 4      # index scan, tiles | side gather, forward | Delta, dQ, dK/dV side, dK/dV window
+        self.launches_per_step = 1 + 2 + 4      # index scan | side gather, forward | Delta, dQ, dK/dV side, dK/dV window
 
     def step(self, bufs=None):
         api = self.api
@@ -295,7 +295,7 @@ def kernel_times(wl: Workload, steps: int):
     def avg(sets, i):
         return sum(s[i].elapsed_time(s[i + 1]) for s in sets) / len(sets) / 1e3
     return {
-        "build_index (2 kernels)": avg(isets, 0),
+        "build_index": avg(isets, 0),
         "gather_side_kv": avg(fsets, 0),
         "attn_fwd_kernel": avg(fsets, 1),
         "bwd_delta": avg(bsets, 1),

@@ -6,9 +6,9 @@
 //                 decoupled look-back over the earlier chunks' published totals give every
 //                 position its global count; the block writes cnt, the shifted copy
 //                 lim[i] = cnt[i-n+1], side_pos, and adds its rows' lim values to the kept-pair
-//                 count of the query tiles they fall in.
-//   index_tiles : per query tile metadata from lim's two end rows, closed-form window pairs,
-//                 side_pos tail fill, header.
+//                 count of the query tiles they fall in.  The block that holds a query tile's
+//                 first (last) row also writes that tile's metadata, every block fills its share
+//                 of the unused end of side_pos, one block writes the header: a single kernel.
 // Chunks are handed out by an atomic ticket per sequence, so a block only ever waits on blocks
 // that started before it; the wait is bounded all the same.
 #include <mutex>
@@ -86,18 +86,28 @@ __device__ __forceinline__ void st_chunk_state(unsigned long long* p, uint32_t s
 constexpr int kLookbackSpins = 1 << 22;
 constexpr int kMaxTilesPerChunk = kIdxChunk / kIdxPerThread + 2;  // query tiles of >= 16 rows under one chunk
 
+// Sum of min(i + 1, n) over rows r0..r1.
+__device__ __forceinline__ long long window_pairs(int r0, int r1, int n) {
+  const long long a = r0 + 1LL, bb = r1 + 1LL;
+  const long long k = min(bb, static_cast<long long>(n));
+  const long long ramp = (a <= k) ? (a + k) * (k - a + 1) / 2 : 0;
+  const long long flat = max(0LL, bb - max(a - 1, static_cast<long long>(n)));
+  return ramp + flat * n;
+}
+
 // NS >= 0: compare against the first NS list entries; NS == kSepHashed: look the token up in
 // `tab`; NS == kByPosition: no token ids, positions that are multiples of `interval` are the
 // members (the fixed-interval variant of Section 4.7 / Appendix J).
 constexpr int kSepHashed = -1, kByPosition = -2;
 template <int NS>
-__global__ void __launch_bounds__(kIdxThreads)
+__global__ void __launch_bounds__(kIdxThreads, 6)
 index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neighbor, SepIds sep,
            const __grid_constant__ SepTable tab,
            unsigned long long* __restrict__ chunk_state, int32_t* __restrict__ tickets,
            int n_chunks, int side_cap, int32_t* __restrict__ cnt, int32_t* __restrict__ lim,
            int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
-           int32_t* __restrict__ tile_meta, int T, int BM, int interval, int32_t* status) {
+           int32_t* __restrict__ tile_meta, int T, int BM, int BN, int interval,
+           const __grid_constant__ sepllm_index_header hdr, int32_t* status) {
   __shared__ int warp_buf[kIdxThreads / 32];
   __shared__ int s_chunk, s_off;
   // counts of the chunk, one pad word per 32 so that a thread's 16 consecutive words and a
@@ -277,31 +287,74 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
       }
     }
   }
-  // side pairs of the query tiles under this chunk's rows: relative sums plus off per row
+  // Query tiles under this chunk's rows: side pairs (relative sums plus off per row) into word 6,
+  // and the rest of the metadata by whoever holds the tile's first row (words 0, 2-5, the window's
+  // share of word 6) or last row (word 1).  tile_meta was zeroed before the launch.
+  int32_t* meta_b = tile_meta + static_cast<size_t>(b) * T * 8;
+  auto window_words = [&](int t) {
+    const int r0 = t * BM, r1 = min(L, (t + 1) * BM) - 1;
+    const int win_lo = max(0, r0 - n_neighbor + 1), win_hi = r1 + 1;
+    int32_t* m = meta_b + static_cast<size_t>(t) * 8;
+    m[2] = win_lo;
+    m[3] = win_hi;
+    m[4] = win_lo / BN;
+    m[5] = (win_hi + BN - 1) / BN;
+    atomicAdd(&m[6], int(window_pairs(r0, r1, n_neighbor)));
+  };
   if (n_rows > 0) {
-    int32_t* meta_b = tile_meta + static_cast<size_t>(b) * T * 8;
     const long long row_hi = row_lo + n_rows;  // exclusive
     const int t_last = int((row_hi - 1) / BM);
-    if (fast_pairs) {
-      for (int t = t_first + tid; t <= t_last; t += kIdxThreads) {
-        const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
-        const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
-        const int sum = tile_part[t - t_first] + off * int(r1 - r0);
-        if (sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
-      }
-    } else {
-      for (int t = t_first + wid; t <= t_last; t += kIdxThreads / 32) {
-        const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
-        const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
-        int sum = 0;
+    for (int t = t_first + (fast_pairs ? tid : wid); t <= t_last; t += (fast_pairs ? kIdxThreads : kIdxThreads / 32)) {
+      const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
+      const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
+      int sum;
+      if (fast_pairs) {
+        sum = tile_part[t - t_first] + off * int(r1 - r0);
+      } else {
+        sum = 0;
         for (long long r = r0 + lane; r < r1; r += 32) {
           const int p = int(r - row_lo);
           sum += cnt_s[p + (p >> 5)] + off;
         }
         sum = warp_sum(sum);
-        if (lane == 0 && sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
+      }
+      if ((fast_pairs || lane == 0)) {
+        if (sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
+        const long long first = static_cast<long long>(t) * BM;
+        const long long last = min(static_cast<long long>(L), first + BM) - 1;
+        if (first >= row_lo) {  // this chunk holds the tile's first row
+          const int p = int(first - row_lo);
+          meta_b[size_t(t) * 8 + 0] = (cnt_s[p + (p >> 5)] + off) / BN;
+          window_words(t);
+        }
+        if (last < row_hi) {    // ... and / or its last row
+          const int p = int(last - row_lo);
+          meta_b[size_t(t) * 8 + 1] = (cnt_s[p + (p >> 5)] + off + BN - 1) / BN;
+        }
       }
     }
+  }
+  if (chunk == 0) {
+    // tiles whose first row comes before row n_neighbor-1 belong to no chunk (lim is 0 there)
+    const int t_head = int(min(static_cast<long long>(T), (static_cast<long long>(shift) + BM - 1) / BM));
+    for (int t = tid; t < t_head; t += kIdxThreads) window_words(t);
+    if (b == 0) {
+      // header: everything but the status word, which any block may be setting
+      const int32_t* src = reinterpret_cast<const int32_t*>(&hdr);
+      int32_t* dst = status;
+      for (int k = 1 + tid; k < int(sizeof(hdr) / 4); k += kIdxThreads) dst[k] = src[k];
+    }
+  }
+  // side_pos beyond n_side reads -1.  If every token after this chunk were a side member the list
+  // would end at `bound`; the previous chunk's bound is higher by this chunk's non-members, and
+  // that stretch is this block's to fill (chunk 0 fills from its bound to the end of the list).
+  {
+    const long long end = min(static_cast<long long>(L), static_cast<long long>(base) + kIdxChunk);
+    const long long bound = off + total + (L - end);
+    const long long upper = (chunk == 0) ? side_cap : min(static_cast<long long>(side_cap),
+                                                          static_cast<long long>(off) + (L - base));
+    int32_t* sp = side_pos + static_cast<size_t>(b) * side_cap;
+    for (long long r = bound + tid; r < upper; r += kIdxThreads) sp[r] = -1;
   }
   if (chunk == n_chunks - 1 && tid == 0) {
     cnt_b[L] = off + total;
@@ -309,55 +362,6 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   }
 }
 
-// Sum of min(i + 1, n) over rows r0..r1.
-__device__ __forceinline__ long long window_pairs(int r0, int r1, int n) {
-  const long long a = r0 + 1LL, bb = r1 + 1LL;
-  const long long k = min(bb, static_cast<long long>(n));
-  const long long ramp = (a <= k) ? (a + k) * (k - a + 1) / 2 : 0;
-  const long long flat = max(0LL, bb - max(a - 1, static_cast<long long>(n)));
-  return ramp + flat * n;
-}
-
-__global__ void __launch_bounds__(256)
-index_tiles(sepllm_index_header hdr, uint8_t* __restrict__ index) {
-  const int B = hdr.desc.B, L = hdr.desc.L, n = hdr.desc.n_neighbor;
-  const int BM = hdr.desc.BM, BN = hdr.desc.BN, T = hdr.n_tiles, side_cap = hdr.desc.side_cap;
-  const int32_t* lim = reinterpret_cast<const int32_t*>(index + hdr.off_lim);
-  const int32_t* n_side = reinterpret_cast<const int32_t*>(index + hdr.off_n_side);
-  int32_t* side_pos = reinterpret_cast<int32_t*>(index + hdr.off_side_pos);
-  int32_t* tile_meta = reinterpret_cast<int32_t*>(index + hdr.off_tile_meta);
-  const int gt = blockIdx.x * blockDim.x + threadIdx.x;
-  const int n_threads = gridDim.x * blockDim.x;
-
-  if (gt == 0) {
-    // everything but the status word, which the scan kernel may have set
-    sepllm_index_header* out = reinterpret_cast<sepllm_index_header*>(index);
-    const int32_t st = out->status;
-    *out = hdr;
-    out->status = st;
-  }
-
-  // one thread per query tile; word 6 already holds the tile's side pairs
-  for (long long u = gt; u < static_cast<long long>(B) * T; u += n_threads) {
-    const int b = int(u / T), t = int(u % T);
-    const int32_t* lim_b = lim + static_cast<size_t>(b) * L;
-    const int r0 = t * BM;
-    const int r1 = min(L, (t + 1) * BM) - 1;
-    int32_t* m = tile_meta + static_cast<size_t>(u) * 8;
-    const int win_lo = max(0, r0 - n + 1), win_hi = r1 + 1;
-    const int side_pairs = m[6];
-    *reinterpret_cast<int4*>(m) = make_int4(lim_b[r0] / BN, (lim_b[r1] + BN - 1) / BN, win_lo, win_hi);
-    *reinterpret_cast<int4*>(m + 4) = make_int4(win_lo / BN, (win_hi + BN - 1) / BN,
-                                                side_pairs + int(window_pairs(r0, r1, n)), 0);
-  }
-
-  // side_pos beyond n_side reads -1
-  for (int b = 0; b < B; ++b) {
-    const int ns = min(n_side[b], side_cap);
-    for (int r = ns + gt; r < side_cap; r += n_threads)
-      side_pos[static_cast<size_t>(b) * side_cap + r] = -1;
-  }
-}
 
 static sepllm_status check_index_desc(const sepllm_index_desc* d) {
   if (!d) return SEPLLM_INVALID_ARG;
@@ -422,8 +426,8 @@ static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_in
       reinterpret_cast<int32_t*>(blob + h.off_lim),                                              \
       reinterpret_cast<int32_t*>(blob + h.off_side_pos),                                         \
       reinterpret_cast<int32_t*>(blob + h.off_n_side),                                           \
-      reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM, interval,         \
-      reinterpret_cast<int32_t*>(blob))
+      reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM, desc->BN,         \
+      interval, h, reinterpret_cast<int32_t*>(blob))
   SepTable tab;
   tab.mult = 0;
   const bool hashed = sep.n > 0 && build_sep_table(sep_ids, sep.n, &tab);
@@ -436,9 +440,6 @@ static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_in
   else if (sep.n <= 32) SEPLLM_SCAN(32);
   else SEPLLM_SCAN(64);
 #undef SEPLLM_SCAN
-  const long long units = static_cast<long long>(desc->B) * h.n_tiles;
-  const int blocks = int(max(1LL, min(148LL * 8, (units + 255) / 256)));
-  index_tiles<<<blocks, 256, 0, stream>>>(h, blob);
   SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }

@@ -25,6 +25,10 @@
  *        Q, O, dO, dQ : [B][Hq][L][d]        K, V, dK, dV : [B][Hkv][L][d]
  *        LSE          : [B][Hq][L] fp32, natural logarithm
  *    Query head h reads KV head h / (Hq/Hkv).
+ *  - Sequences shorter than L are padded at the end (any token ids, any finite
+ *    K, V, Q values): the mask is causal, so no valid row sees a padded key,
+ *    and with dO = 0 on the padded rows the padded queries add nothing to dK
+ *    and dV.  Outputs of padded rows are to be ignored.
  *  - Supported: d in {64, 128}; Hq a multiple of Hkv; n_neighbor >= 1;
  *    n_init >= 0; index tiles BM = BN = 128 for the attention calls.
  */

@@ -154,8 +154,8 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
  * without ordering, or different host threads) race on it and must be
  * serialised by the caller.  The array keeps the last call's contents; each
  * call clears the words it is going to use (a memset on `stream`, before its
- * kernels), so back-to-back calls are independent.  Other arguments and the written index are exactly those of
- * sepllm_build_index. */
+ * kernel), so back-to-back calls are independent.  Other arguments and the
+ * written index are exactly those of sepllm_build_index. */
 sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* sep_ids, void* index, void* stream);
 

@@ -84,7 +84,8 @@ typedef struct {
 } sepllm_attn_desc;
 
 /* Streaming cache capacities in the paper's names (Section 3.3): a initial,
- * s separator, w local window, c total; a + s + w < c, w >= 1. */
+ * s separator, w local window, c total; a + s + w < c, w >= 1.  The cache
+ * calls take up to 16 query heads per kv head (Hq / Hkv <= 16). */
 typedef struct {
   int32_t B, Hkv, Hq, d, a, s, w, c;
 } sepllm_cache_desc;

@@ -35,7 +35,7 @@ static sepllm_status fill_cache_header(const sepllm_cache_desc* d, sepllm_cache_
   if (!(static_cast<int64_t>(d->a) + d->s + d->w < d->c)) return SEPLLM_INVALID_ARG;
   if (d->Hq % d->Hkv != 0) return SEPLLM_INVALID_ARG;
   if (d->d != 64 && d->d != 128) return SEPLLM_UNSUPPORTED;
-  if (d->Hq / d->Hkv > 8) return SEPLLM_UNSUPPORTED;
+  if (d->Hq / d->Hkv > 16) return SEPLLM_UNSUPPORTED;
   *h = sepllm_cache_header{};
   h->magic = SEPLLM_CACHE_MAGIC;
   h->version = 1;
@@ -504,7 +504,11 @@ constexpr int decode_smem_bytes() {
 // position inside the cache, entry v of the walk above at position v) and q arrives un-rotated:
 // it is rotated to position Size_run - 1, pair (i, i + D/2) by the angle (Size_run - 1) * theta_i
 // from a table of (cos, sin) per (position, i), while its fragments load.
-template <int D, bool ROPE>
+//
+// WIDE: groups of 9 to 16 query heads per kv head use both row halves of the MMA tile (a lane
+// then carries the softmax state of rows frow and frow + 8); narrower groups leave the upper
+// half zero and skip its arithmetic.
+template <int D, bool ROPE, bool WIDE>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
              const uint8_t* __restrict__ state, const __nv_bfloat16* __restrict__ Kc,
@@ -515,6 +519,8 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   constexpr int TILEB = kDecTile * ROWB;    // bytes of one K (or V) tile
   constexpr int NW = kDecThreads / 32;
   constexpr int RPP = 32 / CH;              // rows covered by one pass of the warp's copies
+  constexpr int RH = WIDE ? 2 : 1;          // row halves of the 16-row MMA tile in use
+  constexpr int GS = 8 * RH;                // rows per warp in the merge buffers
   extern __shared__ __align__(128) uint8_t dec_smem[];
   const sepllm_cache_desc d = h.desc;
   const int G = d.Hq / d.Hkv;
@@ -538,9 +544,9 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   const int frow = lane >> 2, fcol = (lane & 3) * 2;
   uint32_t qa[D / 16][4];
   {
-    const __nv_bfloat16* qrow = q_in + (size_t(b) * d.Hq + hk * G + min(frow, G - 1)) * D;
-    // two consecutive elements e, e+1 of the (rotated) query row as packed bf16
-    auto q_pair = [&](int e) -> uint32_t {
+    // two consecutive elements e, e+1 of the (rotated) query row `row` as packed bf16
+    auto q_pair = [&](int row, int e) -> uint32_t {
+      const __nv_bfloat16* qrow = q_in + (size_t(b) * d.Hq + hk * G + min(row, G - 1)) * D;
       if (!ROPE) return *reinterpret_cast<const uint32_t*>(qrow + e);
       const int i = e % (D / 2);
       const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qrow + e));
@@ -552,10 +558,11 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
     };
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-      qa[ks][0] = (frow < G && size_run > 0) ? q_pair(ks * 16 + fcol) : 0u;
-      qa[ks][2] = (frow < G && size_run > 0) ? q_pair(ks * 16 + 8 + fcol) : 0u;
-      qa[ks][1] = 0u;
-      qa[ks][3] = 0u;
+      const bool lo = frow < G && size_run > 0, hi = WIDE && frow + 8 < G && size_run > 0;
+      qa[ks][0] = lo ? q_pair(frow, ks * 16 + fcol) : 0u;
+      qa[ks][2] = lo ? q_pair(frow, ks * 16 + 8 + fcol) : 0u;
+      qa[ks][1] = hi ? q_pair(frow + 8, ks * 16 + fcol) : 0u;
+      qa[ks][3] = hi ? q_pair(frow + 8, ks * 16 + 8 + fcol) : 0u;
     }
   }
 
@@ -583,7 +590,10 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   for (int n = 0; n < D / 8; ++n)
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[n][e] = 0.f;
-  float m_ref = -INFINITY, l_part = 0.f;  // of row `frow`; l_part is this lane's share of the sum
+  // of rows frow (+ 8): reference exponent and this lane's share of the row sum
+  float m_ref[RH], l_part[RH];
+#pragma unroll
+  for (int r = 0; r < RH; ++r) { m_ref[r] = -INFINITY; l_part[r] = 0.f; }
 
 #pragma unroll
   for (int s = 0; s < kDecStages - 1; ++s) {
@@ -614,39 +624,43 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
         mma_16816(sc[1], qa[ks], kb[2], kb[3]);
       }
     }
-    // online softmax over the 16 rows of the tile for query head `frow`
+    // online softmax over the 16 cache rows of the tile for query heads frow (and frow + 8)
     const int vbase = v0 + (wid + i * NW) * kDecTile;
-    float sv[4];
-#pragma unroll
-    for (int n = 0; n < 2; ++n)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int v = vbase + n * 8 + fcol + e;
-        sv[n * 2 + e] = (v < v1) ? sc[n][e] * scale_log2 : -INFINITY;
-      }
-    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    float corr = 1.f;
+    uint32_t pa[4] = {0u, 0u, 0u, 0u};
+    float corr[RH];
     bool rescale = false;
-    if (mx > m_ref + 8.f) {  // lazy: the reference moves only when the maximum grew by > 2^8
-      corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - mx);
-      m_ref = mx;
-      rescale = true;
+#pragma unroll
+    for (int r = 0; r < RH; ++r) {
+      float sv[4];
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int v = vbase + n * 8 + fcol + e;
+          sv[n * 2 + e] = (v < v1) ? sc[n][2 * r + e] * scale_log2 : -INFINITY;
+        }
+      float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      corr[r] = 1.f;
+      if (mx > m_ref[r] + 8.f) {  // lazy: the reference moves only when the maximum grew by > 2^8
+        corr[r] = (m_ref[r] == -INFINITY) ? 0.f : ex2(m_ref[r] - mx);
+        m_ref[r] = mx;
+        rescale = true;
+      }
+      const float m_eff = (m_ref[r] == -INFINITY) ? 0.f : m_ref[r];
+      const float p0 = ex2(sv[0] - m_eff), p1 = ex2(sv[1] - m_eff);
+      const float p2 = ex2(sv[2] - m_eff), p3 = ex2(sv[3] - m_eff);
+      l_part[r] = l_part[r] * corr[r] + (p0 + p1) + (p2 + p3);
+      pa[r] = pack_bf16(p0, p1);
+      pa[2 + r] = pack_bf16(p2, p3);
     }
-    const float m_eff = (m_ref == -INFINITY) ? 0.f : m_ref;
-    const float p0 = ex2(sv[0] - m_eff), p1 = ex2(sv[1] - m_eff);
-    const float p2 = ex2(sv[2] - m_eff), p3 = ex2(sv[3] - m_eff);
-    l_part = l_part * corr + (p0 + p1) + (p2 + p3);
     if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-      for (int n = 0; n < D / 8; ++n) { oacc[n][0] *= corr; oacc[n][1] *= corr; }
+      for (int n = 0; n < D / 8; ++n)
+#pragma unroll
+        for (int r = 0; r < RH; ++r) { oacc[n][2 * r] *= corr[r]; oacc[n][2 * r + 1] *= corr[r]; }
     }
-    uint32_t pa[4];
-    pa[0] = pack_bf16(p0, p1);
-    pa[1] = 0u;
-    pa[2] = pack_bf16(p2, p3);
-    pa[3] = 0u;
     // O[16 heads x D] += P V
     {
       const int key = (lane & 7) + (((lane >> 3) & 1) << 3);
@@ -662,33 +676,40 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
     __syncwarp();  // every lane is done with this stage before a later copy overwrites it
   }
   cp_async_wait<0>();
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
-  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+#pragma unroll
+  for (int r = 0; r < RH; ++r) {
+    l_part[r] += __shfl_xor_sync(0xffffffffu, l_part[r], 1);
+    l_part[r] += __shfl_xor_sync(0xffffffffu, l_part[r], 2);
+  }
   __syncthreads();  // all warps are out of their stage buffers
 
   // merge the warps' partials: sm_ml[w][g] = (m, l), sm_acc[w][g][D]
   float2* sm_ml = reinterpret_cast<float2*>(dec_smem);
-  float* sm_acc = reinterpret_cast<float*>(dec_smem + NW * 8 * sizeof(float2));
-  if (frow < G) {
-    if ((lane & 3) == 0) sm_ml[wid * 8 + frow] = make_float2(m_ref, l_part);
+  float* sm_acc = reinterpret_cast<float*>(dec_smem + NW * GS * sizeof(float2));
 #pragma unroll
-    for (int n = 0; n < D / 8; ++n)
-      *reinterpret_cast<float2*>(sm_acc + (wid * 8 + frow) * D + n * 8 + fcol) =
-          make_float2(oacc[n][0], oacc[n][1]);
+  for (int r = 0; r < RH; ++r) {
+    const int g = frow + 8 * r;
+    if (g < G) {
+      if ((lane & 3) == 0) sm_ml[wid * GS + g] = make_float2(m_ref[r], l_part[r]);
+#pragma unroll
+      for (int n = 0; n < D / 8; ++n)
+        *reinterpret_cast<float2*>(sm_acc + (wid * GS + g) * D + n * 8 + fcol) =
+            make_float2(oacc[n][2 * r], oacc[n][2 * r + 1]);
+    }
   }
   __syncthreads();
   for (int idx = tid; idx < G * D; idx += kDecThreads) {
     const int g = idx / D, e = idx % D;
     float mm = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sm_ml[w * 8 + g].x);
+    for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sm_ml[w * GS + g].x);
     float ll = 0.f, aa = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
-      const float2 ml = sm_ml[w * 8 + g];
+      const float2 ml = sm_ml[w * GS + g];
       const float scf = (ml.x == -INFINITY) ? 0.f : ex2(ml.x - mm);
       ll += ml.y * scf;
-      aa += sm_acc[(w * 8 + g) * D + e] * scf;
+      aa += sm_acc[(w * GS + g) * D + e] * scf;
     }
     const size_t uo = ((size_t(b) * d.Hq + hk * G + g) * splits + split);
     part_acc[uo * D + e] = aa;
@@ -879,19 +900,31 @@ extern "C" sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* 
   return SEPLLM_OK;
 }
 
-template <int D, bool ROPE>
+template <int D, bool ROPE, bool WIDE>
 static sepllm_status launch_decode(const sepllm_cache_header& h, float scale_log2, const void* q,
                                    const void* state, const void* Kc, const void* Vc, float* ml,
                                    float* acc, int splits, const float2* rope, cudaStream_t stream) {
   constexpr int smem = decode_smem_bytes<D>();
-  static_assert(smem >= (kDecThreads / 32) * 8 * (8 + D * 4), "partials fit in the stage buffers");
-  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D, ROPE>,
+  static_assert(smem >= (kDecThreads / 32) * 16 * (8 + D * 4), "partials fit in the stage buffers");
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D, ROPE, WIDE>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  decode_split<D, ROPE><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
+  decode_split<D, ROPE, WIDE><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
       h, scale_log2, static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(state),
       static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc, splits,
       rope);
   return SEPLLM_OK;
+}
+
+template <int D>
+static sepllm_status dispatch_decode(bool with_rope, bool wide, const sepllm_cache_header& h,
+                                     float scale_log2, const void* q, const void* state,
+                                     const void* Kc, const void* Vc, float* ml, float* acc,
+                                     int splits, const float2* rope, cudaStream_t stream) {
+  if (with_rope)
+    return wide ? launch_decode<D, true, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
+                : launch_decode<D, true, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
+  return wide ? launch_decode<D, false, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
+              : launch_decode<D, false, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
 }
 
 static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, const void* q,
@@ -914,12 +947,10 @@ static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, con
   float* acc = reinterpret_cast<float*>(ws + kAlign + align_up(units * 2 * sizeof(float)));
   if (scale == 0.f) scale = 1.0f / sqrtf(float(desc->d));
   const float scale_log2 = scale * 1.4426950408889634f;
-  if (desc->d == 128)
-    st = rope ? launch_decode<128, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
-              : launch_decode<128, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
-  else
-    st = rope ? launch_decode<64, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
-              : launch_decode<64, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
+  const bool wide = desc->Hq / desc->Hkv > 8;
+  st = (desc->d == 128)
+           ? dispatch_decode<128>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
+           : dispatch_decode<64>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
   if (st != SEPLLM_OK) return st;
   if (desc->d == 128)
     decode_combine<128><<<dim3(desc->Hq, desc->B), 128, 0, stream>>>(

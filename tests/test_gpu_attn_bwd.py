@@ -37,6 +37,16 @@ def test_bwd_shapes(d, Hq, Hkv, L, a, n):
     _run(2, Hq, Hkv, L, d, a, n, 0.15, 200 + L + d)
 
 
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 16, 1), (128, 12, 2), (64, 3, 1)])
+def test_bwd_wide_and_odd_query_groups(d, Hq, Hkv):
+    """16 query heads per kv head (Falcon-40B's ratio), 6, and an odd group of 3 (no head pairing);
+    the forward is checked on the way through the backward's inputs."""
+    (Qd, Kd, Vd, dOd, O, LSE, idesc, index), _ = _run(1, Hq, Hkv, 700, d, 3, 96, 0.2, 230 + Hq)
+    f = flags_of(inputs.token_ids(230 + Hq, 1, 700, 0.2, "iid"), inputs.SEP_IDS)
+    Oref, _ = orc.attn_fwd(Qd.double().cpu().numpy(), Kd.double().cpu().numpy(), Vd.double().cpu().numpy(), f, 3, 96)
+    assert_close(O.float().cpu().numpy(), Oref, dict(max_abs=1e-2, rel_fro=5e-3), "O")
+
+
 def test_bwd_fp32_gradients_and_determinism():
     args, (dQ, dK, dV) = _run(1, 4, 2, 900, 128, 4, 100, 0.2, 71, grad_dtype=1)
     assert dQ.dtype == torch.float32

@@ -101,6 +101,13 @@ def test_cache_small_every_step(d, Hq, Hkv):
     assert min(c.compactions for c in oc) > 10
 
 
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 16, 1), (128, 32, 2), (128, 9, 1), (64, 24, 2)])
+def test_cache_wide_query_groups(d, Hq, Hkv):
+    """9 to 16 query heads per kv head (Falcon-40B has 16 at d = 64): both halves of the decode
+    kernel's 16-row tile are in use."""
+    _drive(2, Hkv, Hq, d, a=2, s=6, w=5, c=40, steps=150, rho=0.3, seed=57 + d + Hq, check_every=7)
+
+
 def test_cache_no_initial_tokens_and_no_separator_cache():
     _drive(1, 1, 1, 64, a=0, s=3, w=2, c=9, steps=80, rho=0.5, seed=61)
     _drive(1, 1, 2, 64, a=3, s=0, w=5, c=12, steps=80, rho=0.5, seed=62)     # StreamingLLM-like
@@ -131,4 +138,7 @@ def test_cache_rejects_bad_capacities():
     assert e.value.code == api.INVALID_ARG
     with pytest.raises(api.SepllmError) as e:
         api.sepllm_cache_bytes(api.CacheDesc(1, 1, 1, 80, 4, 10, 10, 100))
+    assert e.value.code == api.UNSUPPORTED
+    with pytest.raises(api.SepllmError) as e:
+        api.sepllm_cache_bytes(api.CacheDesc(1, 1, 17, 64, 4, 10, 10, 100))     # 17 query heads per kv head
     assert e.value.code == api.UNSUPPORTED

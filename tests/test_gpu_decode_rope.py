@@ -71,7 +71,7 @@ def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at, keys_eve
                     assert abs(ln[b, h] - lref) <= TOL_LSE_ROPE
 
 
-@pytest.mark.parametrize("d,Hq,Hkv", [(64, 2, 2), (128, 8, 2), (128, 4, 1)])
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 2, 2), (128, 8, 2), (128, 4, 1), (64, 16, 1), (128, 12, 1)])
 def test_rope_decode_small(d, Hq, Hkv):
     _drive(2, Hkv, Hq, d, a=2, s=5, w=4, c=20, steps=90, rho=0.3, seed=70 + d + Hq, base=10000.0,
            check_at={0, 1, 5, 19, 20, 21, 47, 89}, keys_every=1)

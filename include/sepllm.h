@@ -160,9 +160,10 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
 sepllm_status sepllm_build_index_static(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* sep_ids, void* index, void* stream);
 
-/* Index of the fixed-interval variant (Section 4.7 "Fixed-Interval Variant",
- * Appendix J: instead of the separators, one token every `interval` positions
- * is attended to between the initial and the neighbouring tokens).  The side
+/* Index of the fixed-interval variant (Section 4.7 and the appendix, both
+ * under "Fixed-Interval Variant": instead of the separators, one token every
+ * `interval` positions is attended to between the initial and the
+ * neighbouring tokens).  The side
  * members are the first n_init positions and every position j with
  * j % interval == 0 (the paper does not say where the intervals start; they
  * start at position 0 here).  No token ids are read; desc->n_sep must be 0,

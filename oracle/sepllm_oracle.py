@@ -48,9 +48,10 @@ def separator_flags(token_ids: np.ndarray, sep_ids: Iterable[int]) -> np.ndarray
 
 
 def fixed_interval_flags(L: int, interval: int) -> np.ndarray:
-    """Flags of the fixed-interval variant (Section 4.7, Appendix J): one token
-    every ``interval`` positions takes the separators' place.  The paper does
-    not say where the intervals start; here they start at position 0."""
+    """Flags of the fixed-interval variant (Section 4.7 and the appendix
+    "Fixed-Interval Variant"): one token every ``interval`` positions takes the
+    separators' place.  The paper does not say where the intervals start; here
+    they start at position 0."""
     return (np.arange(L) % int(interval)) == 0
 
 

@@ -97,7 +97,7 @@ __device__ __forceinline__ long long window_pairs(int r0, int r1, int n) {
 
 // NS >= 0: compare against the first NS list entries; NS == kSepHashed: look the token up in
 // `tab`; NS == kByPosition: no token ids, positions that are multiples of `interval` are the
-// members (the fixed-interval variant of Section 4.7 / Appendix J).
+// members (the fixed-interval variant: Section 4.7 and the appendix "Fixed-Interval Variant").
 constexpr int kSepHashed = -1, kByPosition = -2;
 template <int NS>
 __global__ void __launch_bounds__(kIdxThreads, 6)

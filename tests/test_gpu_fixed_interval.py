@@ -1,4 +1,5 @@
-"""The fixed-interval variant (Appendix J) through the same index and attention kernels."""
+"""The fixed-interval variant (appendix "Fixed-Interval Variant") through the same index and
+attention kernels."""
 import numpy as np
 import pytest
 import torch

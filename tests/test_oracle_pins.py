@@ -46,7 +46,7 @@ def test_mask_matches_set_construction(a, n):
 
 
 def test_fixed_interval_variant_mask():
-    """Appendix J in words: the initial tokens, one token every `interval`
+    """The appendix "Fixed-Interval Variant" in words: the initial tokens, one token every `interval`
     positions, the n closest tokens.  interval = 1 keeps everything (dense
     causal); an interval beyond the length keeps only position 0 besides the
     initial and neighbouring tokens (the StreamingLLM pattern when a >= 1)."""

@@ -544,9 +544,10 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   const int frow = lane >> 2, fcol = (lane & 3) * 2;
   uint32_t qa[D / 16][4];
   {
-    // two consecutive elements e, e+1 of the (rotated) query row `row` as packed bf16
-    auto q_pair = [&](int row, int e) -> uint32_t {
-      const __nv_bfloat16* qrow = q_in + (size_t(b) * d.Hq + hk * G + min(row, G - 1)) * D;
+    // two consecutive elements e, e+1 of a (rotated) query row as packed bf16
+    const __nv_bfloat16* q_lo = q_in + (size_t(b) * d.Hq + hk * G + min(frow, G - 1)) * D;
+    const __nv_bfloat16* q_hi = q_in + (size_t(b) * d.Hq + hk * G + min(frow + 8, G - 1)) * D;
+    auto q_pair = [&](const __nv_bfloat16* qrow, int e) -> uint32_t {
       if (!ROPE) return *reinterpret_cast<const uint32_t*>(qrow + e);
       const int i = e % (D / 2);
       const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qrow + e));
@@ -559,10 +560,10 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
       const bool lo = frow < G && size_run > 0, hi = WIDE && frow + 8 < G && size_run > 0;
-      qa[ks][0] = lo ? q_pair(frow, ks * 16 + fcol) : 0u;
-      qa[ks][2] = lo ? q_pair(frow, ks * 16 + 8 + fcol) : 0u;
-      qa[ks][1] = hi ? q_pair(frow + 8, ks * 16 + fcol) : 0u;
-      qa[ks][3] = hi ? q_pair(frow + 8, ks * 16 + 8 + fcol) : 0u;
+      qa[ks][0] = lo ? q_pair(q_lo, ks * 16 + fcol) : 0u;
+      qa[ks][2] = lo ? q_pair(q_lo, ks * 16 + 8 + fcol) : 0u;
+      qa[ks][1] = hi ? q_pair(q_hi, ks * 16 + fcol) : 0u;
+      qa[ks][3] = hi ? q_pair(q_hi, ks * 16 + 8 + fcol) : 0u;
     }
   }
 

@@ -14,8 +14,13 @@ pytestmark = pytest.mark.gpu
 # The library rounds the rotated K rows and the rotated q to bf16 before the tensor-core products
 # (the oracle rotates in fp64), so every score carries two relative roundings of 2^-9 per term:
 # about 2^-9 * sqrt(2) * |q||k| / d ~ 3e-3 rms for N(0,1) inputs.  LSE is a weighted mean of the
-# scores' errors, hence the looser bound than for the plain decode; O keeps the common tolerance.
+# scores' errors, hence the looser bound than for the plain decode.  Each weight P_j then carries
+# that score error as a relative error of its own (about 2e-3 rms, independent from key to key),
+# which adds to the rounding of P and of the output that the plain decode already has: about 3e-3
+# relative on O as a whole, up to 5e-3 on single heads with few cache entries, so the relative
+# Frobenius bound on O is twice the common one here; the max-abs bound is the common one.
 TOL_LSE_ROPE = 1e-2
+TOL_O_ROPE = dict(max_abs=TOL_O["max_abs"], rel_fro=2 * TOL_O["rel_fro"])
 
 
 def _check_rotated_keys(gc, Kr, st, base):
@@ -67,7 +72,7 @@ def _drive(B, Hkv, Hq, d, a, s, w, c, steps, rho, seed, base, check_at, keys_eve
                     h = hk * G + g
                     oref, lref = orc.decode_attention_rope(qp[t, b, h].double().numpy(), Kc[b, hk][slots],
                                                            Vc[b, hk][slots], base)
-                    assert_close(on[b, h], oref, TOL_O, f"rope decode o t={t} b={b} h={h}")
+                    assert_close(on[b, h], oref, TOL_O_ROPE, f"rope decode o t={t} b={b} h={h}")
                     assert abs(ln[b, h] - lref) <= TOL_LSE_ROPE
 
 

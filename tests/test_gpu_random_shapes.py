@@ -1,0 +1,57 @@
+"""Seeded random shapes through index, forward and backward (lengths that are no tile multiple,
+neighbour counts from 1 to beyond L, separator rates from none to all, odd head groups)."""
+import numpy as np
+import pytest
+
+from oracle import sepllm_oracle as orc
+from paper_2412_12094_b200 import api, inputs
+from tests._gpu_util import TOL_GRAD, TOL_LSE, TOL_O, assert_close, attn_bwd, attn_fwd, build_index, errors, flags_of
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(seed):
+    g = np.random.default_rng(seed)
+    d = int(g.choice([64, 128]))
+    Hkv = int(g.choice([1, 2, 3]))
+    G = int(g.choice([1, 2, 3, 4, 5, 8]))
+    return dict(d=d, Hkv=Hkv, Hq=Hkv * G, B=int(g.choice([1, 2, 3])), L=int(g.integers(1, 1400)),
+                a=int(g.choice([0, 1, 4, 7, 130])), n=int(g.choice([1, 2, 17, 64, 128, 129, 300, 2000])),
+                rho=float(g.choice([0.0, 0.02, 0.1, 0.3, 0.9, 1.0])), gd=int(g.choice([0, 1])))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shape(seed):
+    c = _case(7000 + seed)
+    B, Hq, Hkv, L, d, a, n = c["B"], c["Hq"], c["Hkv"], c["L"], c["d"], c["a"], c["n"]
+    if c["rho"] < 1.0:
+        ids = inputs.token_ids(7000 + seed, B, L, c["rho"])
+    else:
+        ids = np.full((B, L), inputs.SEP_IDS[2], np.int32)
+    f = flags_of(ids, inputs.SEP_IDS)
+    Q, K, V, dO = inputs.qkv_do(7000 + seed, B, Hq, Hkv, L, d)
+    idesc, index = build_index(ids, inputs.SEP_IDS, a, n)
+    got = api.read_index(index)
+    ref = orc.build_index_fast(ids, inputs.SEP_IDS, a, n, 128, 128, L)
+    for k in ("cnt", "lim", "side_pos", "n_side", "tile_meta"):
+        assert np.array_equal(got[k], ref[k]), (k, c)
+    Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
+    O, LSE = attn_fwd(Qd, Kd, Vd, idesc, index)
+    Oref, LSEref = orc.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), f, a, n)
+    assert_close(O.float().cpu().numpy(), Oref, TOL_O, f"O {c}")
+    assert np.abs(LSE.cpu().numpy() - LSEref).max() <= TOL_LSE, c
+    grads = attn_bwd(dOd, Qd, Kd, Vd, O, LSE, idesc, index, grad_dtype=c["gd"])
+    refs = orc.attn_bwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), dO.double().numpy(), f, a, n)
+    for got_g, ref_g, what in zip(grads, refs, ("dQ", "dK", "dV")):
+        got_g = got_g.float().cpu().numpy()
+        # Where a handful of keys collect thousands of weights near 1/8 (n = 1 or 2, no side entries)
+        # gradient entries reach 10 and more and the bf16 rounding of dS, 2^-9 of each term, adds up
+        # in proportion: the absolute bound is taken relative to the tensor's largest entry there.
+        big = max(1.0, float(np.abs(ref_g).max()))
+        diff = np.abs(got_g - ref_g)
+        assert np.isfinite(got_g).all(), (what, c)
+        assert diff.max() <= TOL_GRAD["max_abs"] * big, (what, float(diff.max()), big, c)
+        if np.linalg.norm(ref_g) > 1e-6:      # n = 1 without side entries: every dQ and dK is exactly 0
+            assert errors(got_g, ref_g)[1] <= TOL_GRAD["rel_fro"], (what, errors(got_g, ref_g), c)
+        else:
+            assert diff.max() <= 1e-4, (what, float(diff.max()), c)

@@ -223,40 +223,49 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
       const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);                // K as the K-major B of S
       const uint32_t kt_lo0 = desc_lo(smem_u32(sKV), kTileBlockBytes);  // K as the MN-major B of dQ
-      auto issue_s = [&](int gi) {
-        const uint32_t k_lo = k_lo0 + (gi % NST) * (C::kStage >> 4);
+      // The issuing thread's own scalar instructions sit between the MMAs of consecutive groups
+      // (one warp issues a dependent instruction every few cycles, and the tensor pipe holds next
+      // to no queue), so the loop carries the ring stage and the barrier parities along instead of
+      // dividing tile counters.
+      auto issue_s = [&](int st) {
+        const uint32_t k_lo = k_lo0 + st * (C::kStage >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kS, tmem + C::kQt + k * 8, k_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
         tc_commit(bar_s);
       };
-      auto issue_dp = [&](int gi) {
-        const uint32_t v_lo = k_lo0 + (gi % NST) * (C::kStage >> 4) + (C::kTile >> 4);
+      auto issue_dp = [&](int st) {
+        const uint32_t v_lo = k_lo0 + st * (C::kStage >> 4) + (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ts_lo(tmem + C::kdP, tmem + C::kdOt + k * 8, v_lo + kmajor_step(k, kTileBlockBytes),
                      idesc_s, k > 0);
         tc_commit(bar_dp);
       };
-      int tb = 0, ino = 0;
+      int ino = 0;
+      int st = 0;            // ring stage of the current tile
+      uint32_t fpar = 0;     // parity of that stage's "full" barrier
+      uint32_t gpar = 0;     // parity of the per-tile barriers (tile counter & 1)
       for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++ino) {
         const int n_tiles = dq_item(p, w).n_tiles;
         wait(bar_qdo, ino & 1);
-        wait(bar_f + tb % NST, (tb / NST) & 1);
+        wait(bar_f + st, fpar);
         tc_fence_after();
-        issue_s(tb);
-        issue_dp(tb);
+        issue_s(st);
+        issue_dp(st);
         for (int j = 0; j < n_tiles; ++j) {
-          const int gi = tb + j, st = gi % NST;
+          int st1 = st + 1;
+          uint32_t fpar1 = fpar;
+          if (st1 == NST) { st1 = 0; fpar1 ^= 1u; }
           if (j + 1 < n_tiles) {
             // S of the next tile as soon as this tile's S has been read out
-            wait(bar_f + (gi + 1) % NST, ((gi + 1) / NST) & 1);
-            wait(bar_sl, gi & 1);
+            wait(bar_f + st1, fpar1);
+            wait(bar_sl, gpar);
             tc_fence_after();
-            issue_s(gi + 1);
+            issue_s(st1);
           }
-          wait(bar_ds, gi & 1);
+          wait(bar_ds, gpar);
           if (j == 0 && ino > 0) wait(bar_dqf, (ino - 1) & 1);  // the previous item's dQ is stored
           tc_fence_after();
           // dS of keys [64u, 64u+64) sits in columns 64u .. 64u+31 of the dP range
@@ -266,10 +275,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
             umma_ts_lo(tmem + C::kdQ, tmem + C::kdP + (k >> 2) * 64 + (k & 3) * 8,
                        kt_lo + mnmajor_step(k), idesc_dq, (j > 0 || k > 0));
           tc_commit(bar_e + st);
-          if (j + 1 < n_tiles) issue_dp(gi + 1);
+          if (j + 1 < n_tiles) issue_dp(st1);
+          st = st1;
+          fpar = fpar1;
+          gpar ^= 1u;
         }
         tc_commit(bar_acc);
-        tb += n_tiles;
       }
     }
   } else {

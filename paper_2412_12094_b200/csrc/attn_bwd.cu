@@ -572,53 +572,66 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint32_t q_lo0 = desc_lo(smem_u32(sQ), 16), do_lo0 = desc_lo(smem_u32(sdO), 16);  // K-major B
       const uint32_t qt_lo0 = desc_lo(smem_u32(sQ), kTileBlockBytes);                         // MN-major B
       const uint32_t dot_lo0 = desc_lo(smem_u32(sdO), kTileBlockBytes);
-      auto issue_st = [&](int it) {
-        const uint32_t q_lo = q_lo0 + (it % NSQ) * (C::kTile >> 4);
+      // ring positions and parities are carried along, not divided out of the iteration counter
+      // (the issuing thread's scalar instructions between MMA groups are tensor-pipe idle time)
+      auto issue_st = [&](int sq) {
+        const uint32_t q_lo = q_lo0 + sq * (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ss_lo(tmem + C::kST, k_lo + kmajor_step(k, kTileBlockBytes),
                      q_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
         tc_commit(bar_st);
       };
-      auto issue_dpt = [&](int it) {
-        wait(bar_of + it % NSO, (it / NSO) & 1);
+      auto issue_dpt = [&](int so, uint32_t opar) {
+        wait(bar_of + so, opar);
         tc_fence_after();
-        const uint32_t do_lo = do_lo0 + (it % NSO) * (C::kTile >> 4);
+        const uint32_t do_lo = do_lo0 + so * (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           umma_ss_lo(tmem + C::kdPT, v_lo + kmajor_step(k, kTileBlockBytes),
                      do_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
         tc_commit(bar_dpt);
       };
+      static_assert(NSO == 2, "the dO ring position is the iteration's parity");
       wait(bar_kv, 0);
       wait(bar_qf, 0);
       tc_fence_after();
       issue_st(0);
-      issue_dpt(0);
+      issue_dpt(0, 0);
+      int sq = 0;          // Q ring stage of iteration `it`
+      uint32_t qpar = 0;   // parity of that stage's "full" barrier
       for (int it = 0; it < n_it; ++it) {
+        const uint32_t ipar = uint32_t(it) & 1u;
+        int sq1 = sq + 1;
+        uint32_t qpar1 = qpar;
+        if (sq1 == NSQ) { sq1 = 0; qpar1 ^= 1u; }
+        const int so = int(ipar);                       // dO ring stage of iteration `it`
+        const uint32_t opar1 = (uint32_t(it + 1) >> 1) & 1u;  // "full" parity of iteration it+1's dO stage
         if (it + 1 < n_it) {
-          wait(bar_qf + (it + 1) % NSQ, ((it + 1) / NSQ) & 1);
-          wait(bar_sl, it & 1);
+          wait(bar_qf + sq1, qpar1);
+          wait(bar_sl, ipar);
           tc_fence_after();
-          issue_st(it + 1);
+          issue_st(sq1);
         }
-        wait(bar_pds, it & 1);
+        wait(bar_pds, ipar);
         tc_fence_after();
         // Within the dP^T range, warpgroup u's columns [64u, 64u+64) hold P^T of its 64 queries
         // in the first 32 and dS^T in the last 32.
-        const uint32_t dot_lo = dot_lo0 + (it % NSO) * (C::kTile >> 4);
-        const uint32_t qt_lo = qt_lo0 + (it % NSQ) * (C::kTile >> 4);
+        const uint32_t dot_lo = dot_lo0 + so * (C::kTile >> 4);
+        const uint32_t qt_lo = qt_lo0 + sq * (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k)
           umma_ts_lo(tmem + C::kdV, tmem + C::kdPT + (k >> 2) * 64 + (k & 3) * 8,
                      dot_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
-        tc_commit(bar_oe + it % NSO);
+        tc_commit(bar_oe + so);
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k)
           umma_ts_lo(tmem + C::kdK, tmem + C::kdPT + (k >> 2) * 64 + 32 + (k & 3) * 8,
                      qt_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
-        tc_commit(bar_qe + it % NSQ);
-        if (it + 1 < n_it) issue_dpt(it + 1);
+        tc_commit(bar_qe + sq);
+        if (it + 1 < n_it) issue_dpt(so ^ 1, opar1);
+        sq = sq1;
+        qpar = qpar1;
       }
       tc_commit(bar_acc);
     } else if (warp >= 2) {

@@ -158,7 +158,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   uint64_t* bar_dp = bars + 5;         //       dP of a tile complete
   uint64_t* bar_dqf = bars + 6;        //       dQ of an item read out of tensor memory (8 warps)
   uint64_t* bar_f = bars + 7;          // [NST] stage full
-  uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete)
+  uint64_t* bar_e = bar_f + NST;       // [NST] stage free (its dQ MMAs are complete; one arithmetic thread arrives)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 2 * NST);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
@@ -274,7 +274,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
           for (int k = 0; k < kBN / 16; ++k)
             umma_ts_lo(tmem + C::kdQ, tmem + C::kdP + (k >> 2) * 64 + (k & 3) * 8,
                        kt_lo + mnmajor_step(k), idesc_dq, (j > 0 || k > 0));
-          tc_commit(bar_e + st);
+          // (the stage is reported free by an arithmetic warp once it sees the next dP complete:
+          // a commit here would cost this thread about 90 cycles of tensor-pipe idle time)
           if (j + 1 < n_tiles) issue_dp(st1);
           st = st1;
           fpar = fpar1;
@@ -367,6 +368,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         // phase B: dS = P (dP - Delta)
         wait(bar_dp, gi & 1);
         tc_fence_after();
+        // MMAs complete in issue order and dQ of the tile before this one (of this item or the
+        // last of the previous one) was issued before this dP: its K/V stage is free
+        if (tid == 128 && gi > 0) mbar_arrive(bar_e + (gi - 1) % NST);
         uint32_t pk[32];
         const unsigned long long ndelta2 = pack_f32x2(-delta_i, -delta_i);
 #pragma unroll

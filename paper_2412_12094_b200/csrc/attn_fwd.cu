@@ -190,6 +190,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // When the two slots are the two heads of one query tile they walk the same key tiles, and a
+  // softmax thread of slot 1 can report the K and V stages free (a commit costs the MMA thread
+  // about 90 cycles during which the tensor pipe has nothing queued).
+  const bool free_by_softmax = p.pair_heads && g0.t >= 0 && g1.t >= 0;
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (!mbar_wait(bar, parity, abort_flag)) {
@@ -270,8 +274,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tc_commit(bar_s + x);
           }
         }
-        if (s < n_tiles) tc_commit(bar_ke + s % NST);      // every S MMA reading K(s) is issued
-        if (s >= 1) tc_commit(bar_ve + (s - 1) % NST);     // every PV MMA reading V(s-1) is issued
+        if (!free_by_softmax) {
+          if (s < n_tiles) tc_commit(bar_ke + s % NST);      // every S MMA reading K(s) is issued
+          if (s >= 1) tc_commit(bar_ve + (s - 1) % NST);     // every PV MMA reading V(s-1) is issued
+        }
       }
       tc_commit(bar_o);
     }
@@ -298,6 +304,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         if (!slot_active(g, ns, wlo, j)) continue;
         wait(bar_s + x, n_done & 1);
         tc_fence_after();
+        // MMAs complete in issue order: S of slot 1 for tile j done means both slots' S MMAs have
+        // read K(j) and both PV MMAs have read V(j-1)
+        if (free_by_softmax && tid == 256) {
+          mbar_arrive(bar_ke + j % NST);
+          if (j >= 1) mbar_arrive(bar_ve + (j - 1) % NST);
+        }
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, sreg[c]);
         tmem_ld_wait();

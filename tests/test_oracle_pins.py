@@ -45,6 +45,18 @@ def test_mask_matches_set_construction(a, n):
     assert (orc.mask_rows(f, a, n, rows) == M[rows]).all()
 
 
+def test_mask_regression_golden_ten_tokens():
+    """Not a value of the paper (its mask figure is an image): the ten-token mask as written out
+    by tests/golden/make_mask_golden.py, read back and checked by hand against Section 3.1 (row 9
+    keeps token 0, the separators 3 and 7, and tokens 8, 9)."""
+    sys_path = os.path.join(GOLD, "mask_10_tokens.txt")
+    rows = [l.strip() for l in open(sys_path) if l.strip() and not l.startswith("#")]
+    f = np.array([0, 0, 0, 1, 0, 0, 0, 1, 0, 0], dtype=bool)
+    M = orc.mask_matrix(f, 1, 2)
+    assert ["".join("1" if x else "." for x in r) for r in M] == rows
+    assert rows[9] == "1..1...111" and rows[4] == "1..11....." and rows[0] == "1........."
+
+
 def test_fixed_interval_variant_mask():
     """The appendix "Fixed-Interval Variant" in words: the initial tokens, one token every `interval`
     positions, the n closest tokens.  interval = 1 keeps everything (dense

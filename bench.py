@@ -100,9 +100,11 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(cfg, heads: int, prefix: int):
+def oracle_sample(cfg, heads: int, prefix: int, keep: dict | None = None):
     """Times the fp64 oracle (forward + backward) on the first `prefix` tokens of `heads`
-    query heads of the workload; returns (effective TFLOP/s, seconds, cores, description)."""
+    query heads of the workload; returns (effective TFLOP/s, seconds, cores, description).
+    keep: if given, receives the oracle's dQ of head 0 on those tokens (rows of dQ depend on
+    their own row only, and the mask is causal, so they are also rows of the full problem)."""
     from threadpoolctl import threadpool_info
     from oracle import sepllm_oracle as orc
     L = min(prefix, cfg["L"])
@@ -118,8 +120,12 @@ def oracle_sample(cfg, heads: int, prefix: int):
     t0 = time.perf_counter()
     M = orc.mask_matrix(f, cfg["n_init"], cfg["n_neighbor"])
     for h in range(heads):
-        orc.attn_bwd_head(Q[h], K[h // G], V[h // G], dO[h], M)
+        dq, _, _ = orc.attn_bwd_head(Q[h], K[h // G], V[h // G], dO[h], M)
+        if keep is not None and h == 0:
+            keep["dQ"] = dq
     dt = time.perf_counter() - t0
+    if keep is not None:
+        keep["O"], keep["LSE"], _ = orc.attn_fwd_rows(Q[0], K[0], V[0], M)    # untimed
     cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     tflops = 14.0 * d * pairs * heads / dt / 1e12
     return tflops, dt, cores, f"fwd+bwd of {heads} query head(s) on the first {L} tokens of the workload"
@@ -127,9 +133,10 @@ def oracle_sample(cfg, heads: int, prefix: int):
 
 # ---------------------------------------------------------------------------- GPU arm
 class Workload:
-    def __init__(self, name: str, rank: int, device: torch.device):
+    def __init__(self, name: str, rank: int, device: torch.device, fwd_only: bool = False):
         from paper_2412_12094_b200 import api
         self.api = api
+        self.fwd_only = fwd_only
         cfg = dict(inputs.CONFIGS[name])
         cfg["seed"] = cfg["seed"] + 1000 * rank
         self.cfg, self.name, self.device = cfg, name, device
@@ -139,7 +146,10 @@ class Workload:
         self.host = [t.pin_memory() for t in (Q, K, V, dO)]
         self.ids = self.ids_h.to(device)
         self.Q, self.K, self.V, self.dO = (t.to(device) for t in self.host)
-        self.idesc = api.IndexDesc(B, L, cfg["n_init"], cfg["n_neighbor"], len(inputs.SEP_IDS), 128, 128, L)
+        # capacity of the side list: initial tokens plus separators at 1.25x the expected rate and a
+        # margin (the index reports CAPACITY_EXCEEDED if a sequence has more, and the run stops)
+        side_cap = min(L, (int(1.25 * cfg["rho"] * L) + cfg["n_init"] + 2048 + 127) // 128 * 128)
+        self.idesc = api.IndexDesc(B, L, cfg["n_init"], cfg["n_neighbor"], len(inputs.SEP_IDS), 128, 128, side_cap)
         ib, sb = api.sepllm_index_bytes(self.idesc)
         self.index = api.alloc_bytes(ib)
         self.scratch = api.alloc_bytes(sb)
@@ -154,7 +164,8 @@ class Workload:
         self.dK = torch.empty_like(self.K)
         self.dV = torch.empty_like(self.V)
         self.out_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (self.O, self.dQ, self.dK, self.dV)]
-        self.launches_per_step = 1 + 2 + 4      # index scan | side gather, forward | Delta, dQ, dK/dV side, dK/dV window
+        # index scan | side gather, forward | Delta, dQ, dK/dV side, dK/dV window
+        self.launches_per_step = 1 + 2 + (0 if fwd_only else 4)
 
     def step(self, bufs=None):
         api = self.api
@@ -162,7 +173,8 @@ class Workload:
             self.ids, self.Q, self.K, self.V, self.dO, self.O, self.dQ, self.dK, self.dV)
         api.sepllm_build_index(self.idesc, ids, inputs.SEP_IDS, self.index, self.scratch)
         api.sepllm_attn_fwd(self.fdesc, self.idesc, Q, K, V, self.index, O, self.LSE, self.ws)
-        api.sepllm_attn_bwd(self.bdesc, self.idesc, dO, Q, K, V, O, self.LSE, self.index, dQ, dK, dV, self.ws)
+        if not self.fwd_only:
+            api.sepllm_attn_bwd(self.bdesc, self.idesc, dO, Q, K, V, O, self.LSE, self.index, dQ, dK, dV, self.ws)
 
     # End to end: every step copies its inputs from pinned host memory and its results back.  The
     # copies run on streams of their own over two sets of device buffers, so the copy-in of step
@@ -303,6 +315,29 @@ def kernel_times(wl: Workload, steps: int):
         "bwd_dkv_kernel<side>": avg(bsets, 3),
         "bwd_dkv_kernel<window>": avg(bsets, 4),
     }
+
+
+def bench_other_workloads(main_name, device, peaks, steps=10, warmup=3):
+    """The remaining training / prefill workloads, each timed like the main one (device-resident
+    inputs, index build inside the step).  The prefill-shaped workload is forward only."""
+    out = {}
+    for name in ("tiny", "pythia160m", "llama8b_prefill", "llama8b_long_r05", "llama8b_long_r10", "llama8b_long_r20"):
+        if name == main_name:
+            continue
+        cfg = inputs.CONFIGS[name]
+        fwd_only = name == "llama8b_prefill"
+        wl = Workload(name, 0, device, fwd_only=fwd_only)
+        wl.step()
+        pairs, _ = wl.kept_pairs()
+        sec = timed(wl.step, steps, warmup, lambda: None)
+        flops = (4.0 if fwd_only else 14.0) * cfg["d"] * pairs * cfg["Hq"]
+        tf = flops * steps / sec / 1e12
+        out[name] = {"pass": "fwd" if fwd_only else "fwd+bwd", "ms_per_step": sec / steps * 1e3,
+                     "tflops": tf, "frac_of_bf16_peak": tf / peaks["bf16_tflops_sustained"],
+                     "kept_pairs": pairs, "steps": steps, "gpu_launches": wl.launches_per_step * steps}
+        del wl
+        torch.cuda.empty_cache()
+    return out
 
 
 def bench_decode(device, peaks, steps=4096, rope=False):
@@ -571,10 +606,10 @@ def main():
     side_iters = wl.side_iters
     dom = max(kflops, key=lambda k: kt[k])
     ach = kflops[dom] / kt[dom] / 1e12
-    # DRAM bytes of the dominant kernel: one ncu capture of the 16k-token copy of this workload
-    # (profiles/ncu_full_attention_kernels_llama8b_L16k.md: 811.0 MB read + 34.4 MB written over
-    # 836 side-pass iterations per query head), scaled by iterations, which is what its Q / dO
-    # stream grows with.  Valid for bwd_dkv_kernel<side> as captured; None for anything else.
+    # DRAM bytes of the dominant kernel: from one ncu capture of the 16 384-token copy of this
+    # workload (bytes read + written over 836 side-pass iterations per query head), scaled by the
+    # iteration count, which is what the kernel's Q / dO stream grows with.  Valid for
+    # bwd_dkv_kernel<side> as captured; None for anything else.
     traffic = None
     if dom == "bwd_dkv_kernel<side>" and cfg["d"] == 128 and cfg["Hq"] == 32 and cfg["B"] == 1:
         traffic = (821.90e6 + 38.00e6) * side_iters / 836.0
@@ -594,16 +629,30 @@ def main():
                       "ms_per_step": sec_e / n_e * 1e3, "steps": n_e,
                       "copies": "on their own streams over two sets of device buffers, overlapping the kernels"}
         if rank == 0:
+            # rows of the last step's results that the CPU leg below recomputes (head 0, first tokens)
+            P = min(args.cpu_prefix, cfg["L"])
+            torch.cuda.synchronize()
+            got = {"O": wl.O[0, 0, :P].float().cpu().numpy(), "LSE": wl.LSE[0, 0, :P].cpu().numpy(),
+                   "dQ": wl.dQ[0, 0, :P].float().cpu().numpy()}
             del wl
             torch.cuda.empty_cache()
+            out["workloads"] = bench_other_workloads(args.workload, device, peaks)
             out["decode"] = bench_decode(device, peaks)
             out["decode_rope"] = bench_decode(device, peaks, rope=True)
             out["index"] = bench_index_stream(device, peaks)
             out["hand_off"] = bench_hand_off(device, peaks)
             if world == 1:
-                v, dt, cores, what = oracle_sample(cfg, args.cpu_heads, args.cpu_prefix)
+                keep = {}
+                v, dt, cores, what = oracle_sample(cfg, args.cpu_heads, args.cpu_prefix, keep)
                 out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                        "sample": what, "seconds": dt}
+                # the same rows from the timed GPU run against the oracle's (query head 0)
+                out["parity"] = {"sample": f"O, LSE, dQ of query head 0, first {P} rows, against the fp64 oracle"}
+                for k in ("O", "dQ"):
+                    diff = got[k].astype(np.float64) - keep[k]
+                    out["parity"][k] = {"max_abs": float(np.abs(diff).max()),
+                                        "rel_fro": float(np.linalg.norm(diff) / np.linalg.norm(keep[k]))}
+                out["parity"]["LSE"] = {"max_abs": float(np.abs(got["LSE"] - keep["LSE"]).max())}
     if world > 1:
         barrier()
         dist.destroy_process_group()

@@ -66,8 +66,10 @@ typedef struct {
  * for dQ, dK, dV.
  * flags: SEPLLM_ATTN_SIDE_READY = the workspace already holds the side K/V rows
  *   gathered from these K, V by an earlier attention call on the same workspace
- *   (a backward given the forward's workspace); the call then skips its gather.
- * events / n_events: optional host array of cudaEvent_t handles (NULL / 0 = off).
+ *   (a backward given the forward's workspace); the call then skips its gather
+ *   and leaves the workspace's status word as the earlier call left it.
+ * events / n_events: a measurement aid, not part of the operation: optional host
+ *   array of cudaEvent_t handles (NULL / 0 = off, the normal use).
  *   The call records events[0] on `stream` before its first launch and
  *   events[i] after its i-th launch, for as many as the array holds, so a
  *   caller can time each kernel.  Forward launches: 1 side gather, 2 attention.
@@ -145,12 +147,14 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
  * The scratch lives in a fixed 256 KB array (65536 words) inside the library
  * image, present on every device that loads the library until the process
  * exits.  A call needs two words per 4096-token chunk plus one per sequence,
- * so the limit is B * (2 * ceil(L / 4096) + 1) <= 65536 (for example 32
- * sequences of 4 M ids); beyond it the call returns SEPLLM_BUFFER_TOO_SMALL
- * and launches nothing.  The call itself allocates
- * nothing (no cudaMalloc / cudaFree, no allocating library routine).
- * The first call on each device looks up the array's device address; make that
- * first call outside any stream capture.  All calls on a device share the one
+ * so the limit is B * (2 * ceil(L / 4096) + 1) <= 65536 (for example 31
+ * sequences of 2^22 ids, or 21845 sequences of 4096); beyond it the call
+ * returns SEPLLM_BUFFER_TOO_SMALL and launches nothing.  The call itself
+ * allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ * Every call looks up the array's device address on the current device (a
+ * host-side lookup); the first call on a device also makes the runtime load
+ * the library's kernels there, so make that first call outside any stream
+ * capture.  All calls on a device share the one
  * array: two calls whose kernels may overlap on the GPU (different streams
  * without ordering, or different host threads) race on it and must be
  * serialised by the caller.  The array keeps the last call's contents; each
@@ -269,6 +273,9 @@ sepllm_status sepllm_cache_from_prompt(const sepllm_cache_desc* desc,
                                        void* state, void* Kc, void* Vc, void* Kr,
                                        const void* rope_table, void* stream);
 
+/* The decode workspace holds the per-split partial results; its status word is
+ * always written as 0 (the decode kernels contain no bounded wait and clamp
+ * nothing). */
 sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* desc, size_t* bytes);
 
 /* One query per sequence over every retained entry (Section 3.2 "Generation",

@@ -72,12 +72,13 @@ def mask_matrix(f: np.ndarray, a: int, n: int) -> np.ndarray:
     return causal & (initial | separator | neighbour)
 
 
-def mask_rows(f: np.ndarray, a: int, n: int, rows: np.ndarray) -> np.ndarray:
-    """Rows ``rows`` of the mask of Eq. 2 (same predicate, fewer rows)."""
+def mask_rows(f: np.ndarray, a: int, n: int, rows: np.ndarray, cols: np.ndarray | None = None) -> np.ndarray:
+    """Rows ``rows`` (and, if given, only columns ``cols``) of the mask of Eq. 2: the same
+    predicate on fewer entries."""
     L = f.shape[0]
     i = np.asarray(rows)[:, None]
-    j = np.arange(L)[None, :]
-    return (j <= i) & ((j < a) | f[None, :] | ((i - j) < n))
+    j = (np.arange(L) if cols is None else np.asarray(cols))[None, :]
+    return (j <= i) & ((j < a) | f[j] | ((i - j) < n))
 
 
 def kept_pairs(f: np.ndarray, a: int, n: int) -> int:
@@ -241,6 +242,110 @@ def attn_keys_bwd(Q, K, V, dO, f, a: int, n: int, keys, scale: float | None = No
     dK = (dLam[:, keys].T @ Q[rows]) * scale
     dV = A[:, keys].T @ dO[rows]
     return dK, dV
+
+
+def attn_keys_bwd_blocked(Q, K, V, dO, f, a: int, n: int, keys, scale: float | None = None,
+                          block_rows: int = 1024, with_term_scale: bool = False):
+    """Same result as :func:`attn_keys_bwd` for keys that many rows keep (an
+    initial token or an early separator of a long sequence is kept by every
+    later row, and a dense [rows][L] evaluation of all of them at once does not
+    fit in memory).
+
+    The rows from the first selected key to the end are taken ``block_rows`` at
+    a time.  Within a block only the columns that some row of the block keeps
+    are evaluated: a column that no row of the block keeps has Lambda = -inf,
+    hence weight 0, in every one of those rows, so leaving it out changes
+    nothing.  Each row still sees every key it keeps, so its softmax is the
+    full one of Eq. 1 under the mask of Eq. 2.  The formulas are those of
+    :func:`attn_bwd_head`.  with_term_scale: also return the squares that
+    :func:`attn_bwd_term_scale` sums, for the selected keys (dK, dV, sK2, sV2;
+    the caller adds the squares over the query heads of a group and takes the
+    root).
+    """
+    keys = np.asarray(keys)
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    L, d = Q.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    dK = np.zeros((keys.size, d))
+    dV = np.zeros((keys.size, d))
+    sK2 = np.zeros((keys.size, d))
+    sV2 = np.zeros((keys.size, d))
+    for r0 in range(int(keys.min()), L, block_rows):
+        rows = np.arange(r0, min(L, r0 + block_rows))
+        # columns a row of this block can keep: initial tokens, separators, and the positions
+        # within n of the block; the predicate of Eq. 2 is then evaluated on those columns only
+        j = np.arange(int(rows[-1]) + 1)
+        cols = np.flatnonzero((j < a) | f[j] | (j > r0 - n))
+        M = mask_rows(f, a, n, rows, cols)
+        rows_used = M[:, np.isin(cols, keys)].any(axis=1)
+        if not rows_used.any():
+            continue
+        rows, M = rows[rows_used], M[rows_used]
+        used = M.any(axis=0)                            # every selected key a row keeps is among them
+        cols, M = cols[used], M[:, used]
+        O, _, A = attn_fwd_rows(Q[rows], K[cols], V[cols], M, scale)
+        dA = dO[rows] @ V[cols].T
+        delta = (dO[rows] * O).sum(axis=1, keepdims=True)
+        dLam = A * (dA - delta)
+        where = np.searchsorted(cols, keys)             # column of each selected key inside the block
+        present = (where < cols.size) & (cols[np.minimum(where, cols.size - 1)] == keys)
+        w = where[present]
+        dK[present] += (dLam[:, w].T @ Q[rows]) * scale
+        dV[present] += A[:, w].T @ dO[rows]
+        if with_term_scale:
+            s_delta = np.sqrt(((dO[rows] * O) ** 2).sum(axis=1, keepdims=True))
+            sK2[present] += ((dLam[:, w] ** 2 + (A[:, w] * s_delta) ** 2).T @ (Q[rows] ** 2)) * scale ** 2
+            sV2[present] += (A[:, w] ** 2).T @ (dO[rows] ** 2)
+    if with_term_scale:
+        return dK, dV, sK2, sV2
+    return dK, dV
+
+
+def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None):
+    """Size of the terms behind every gradient entry, for error bounds in tests.
+
+    Each entry of dV, dK, dQ is a sum of products (A_ij dO_i, dLambda_ij Q_i,
+    dLambda_ij K_j).  An implementation that rounds A and dLambda to bf16
+    before its matrix products perturbs every term by up to 2^-9 of its size,
+    independently from term to term, so the error of an entry grows like the
+    root of the sum of its squared terms, not like the entry's own value (which
+    may be small through cancellation).  The backward is also handed O as the
+    bf16 tensor the forward wrote, and rowsum(dO * O) computed from it is off
+    by up to 2^-9 of each product dO_ie O_ie; that error s_i enters dLambda_ij
+    as A_ij s_i, whatever the size of dLambda_ij itself.  Returns the root of
+    the sum of squares of both kinds of terms for dQ [B][Hq][L][d], dK and dV
+    [B][Hkv][L][d] (summed over the query heads that share a KV head, as the
+    gradients are; dV has no term of the second kind)."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    B, Hq, L, d = Q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    sQ = np.zeros((B, Hq, L, d))
+    sK = np.zeros((B, Hkv, L, d))
+    sV = np.zeros((B, Hkv, L, d))
+    for b in range(B):
+        M = mask_matrix(flags[b], a, n)
+        for h in range(Hq):
+            hk = h // G
+            O, _, A = attn_fwd_rows(Q[b, h], K[b, hk], V[b, hk], M, scale)
+            dA = dO[b, h] @ V[b, hk].T
+            delta = (dO[b, h] * O).sum(axis=1, keepdims=True)
+            dLam = A * (dA - delta)
+            s_delta = np.sqrt(((dO[b, h] * O) ** 2).sum(axis=1, keepdims=True))
+            both = dLam ** 2 + (A * s_delta) ** 2
+            sQ[b, h] = both @ (K[b, hk] ** 2) * scale ** 2
+            sK[b, hk] += both.T @ (Q[b, h] ** 2) * scale ** 2
+            sV[b, hk] += (A ** 2).T @ (dO[b, h] ** 2)
+    return np.sqrt(sQ), np.sqrt(sK), np.sqrt(sV)
 
 
 # ----------------------------------------------------------------------------

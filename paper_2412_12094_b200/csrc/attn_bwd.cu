@@ -933,7 +933,9 @@ extern "C" sepllm_status sepllm_attn_bwd(const sepllm_attn_desc* desc,
   if ((st = fill_index_header(idesc, &ih)) != SEPLLM_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
+  // A backward that continues on the forward's workspace keeps the forward's status word: a
+  // condition the forward recorded stays readable until the caller looks at it.
+  if (!(desc->flags & SEPLLM_ATTN_SIDE_READY)) SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
   const uint8_t* idx = static_cast<const uint8_t*>(index);
   if (desc->d == 64)
     return launch_bwd<64>(desc, idesc, ih, dO, Q, K, V, O, LSE, idx, dQ, dK, dV, ws, stream);

@@ -7,6 +7,8 @@
 //                 the Local Window Cache, the older ones the Past Window Cache
 // Decode walks "virtual" entries 0..Size_run-1 = initial, separator (oldest first), neighbour
 // (oldest first) and maps each to its slot, so only retained rows are read.
+#include <algorithm>
+
 #include "attn_common.cuh"
 
 namespace sepllm {
@@ -96,6 +98,17 @@ __device__ __forceinline__ int virtual_to_slot(int v, const sepllm_cache_seq& q,
 }
 
 constexpr int kUpdThreads = 256;
+
+// Writes the header (passed by value, so nothing on the host has to outlive the launch) and zeroes
+// the rest of the state buffer.  grid-stride over 16-byte words; the buffer is 256-byte aligned.
+__global__ void __launch_bounds__(256)
+cache_init_kernel(sepllm_cache_header h, uint4* __restrict__ state, size_t words16) {
+  const uint4* src = reinterpret_cast<const uint4*>(&h);
+  constexpr size_t kHdrWords = sizeof(sepllm_cache_header) / 16;
+  for (size_t k = size_t(blockIdx.x) * blockDim.x + threadIdx.x; k < words16;
+       k += size_t(gridDim.x) * blockDim.x)
+    state[k] = (k < kHdrWords) ? src[k] : make_uint4(0, 0, 0, 0);
+}
 
 // Exclusive rank of every separator among the Past Window entries, in position order.
 // rank_s[k] (k < n_past) = number of separators among past entries [0, k); returns the total.
@@ -787,10 +800,10 @@ extern "C" sepllm_status sepllm_cache_init(const sepllm_cache_desc* desc, void* 
   if (st != SEPLLM_OK) return st;
   if (!state || !aligned(state, kAlign)) return SEPLLM_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(state, 0, size_t(h.total_bytes), stream));
-  SEPLLM_CUDA_TRY(cudaMemcpyAsync(state, &h, sizeof(h), cudaMemcpyHostToDevice, stream));
-  // the header lives on this call's stack: make sure the copy has read it
-  SEPLLM_CUDA_TRY(cudaStreamSynchronize(stream));
+  const size_t words16 = size_t(h.total_bytes) / 16;   // total_bytes is a multiple of 256
+  const unsigned blocks = unsigned(std::min<size_t>((words16 + 255) / 256, 1184));
+  cache_init_kernel<<<blocks, 256, 0, stream>>>(h, static_cast<uint4*>(state), words16);
+  SEPLLM_CUDA_TRY(cudaGetLastError());
   return SEPLLM_OK;
 }
 
@@ -944,6 +957,8 @@ static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, con
   const int splits = decode_splits(desc);
   const size_t units = size_t(desc->B) * desc->Hq * splits;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  // the decode kernels have no bounded waits and report nothing: the status word reads OK
+  SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(int32_t), stream));
   float* ml = reinterpret_cast<float*>(ws + kAlign);
   float* acc = reinterpret_cast<float*>(ws + kAlign + align_up(units * 2 * sizeof(float)));
   if (scale == 0.f) scale = 1.0f / sqrtf(float(desc->d));

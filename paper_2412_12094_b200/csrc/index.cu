@@ -11,8 +11,6 @@
 //                 of the unused end of side_pos, one block writes the header: a single kernel.
 // Chunks are handed out by an atomic ticket per sequence, so a block only ever waits on blocks
 // that started before it; the wait is bounded all the same.
-#include <mutex>
-
 #include "common.cuh"
 
 namespace sepllm {
@@ -491,24 +489,15 @@ extern "C" sepllm_status sepllm_build_index_fixed_interval(const sepllm_index_de
 constexpr int kStaticWords = 65536;
 static __device__ __align__(256) int32_t g_static_chunk_sums[kStaticWords];
 
-constexpr int kMaxDevices = 64;
-static std::mutex g_static_mu;
-static int32_t* g_static_ptr[kMaxDevices] = {};
-
-// Device address of the array on the current device.  The array's name is only a host-side
-// handle here, so the address is looked up once per device and cached.
+// Device address of the array on the current device.  In host code the array's name is only a
+// handle, not an address a kernel could use, so the address is looked up on every call (a
+// host-side table lookup that allocates nothing): nothing is cached that a re-created context
+// could leave dangling.
 static sepllm_status static_chunk_sums(int32_t** out) {
-  int dev = -1;
-  SEPLLM_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return SEPLLM_UNSUPPORTED;
-  std::lock_guard<std::mutex> lock(g_static_mu);
-  if (!g_static_ptr[dev]) {
-    void* p = nullptr;
-    SEPLLM_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_chunk_sums));
-    if (!p) return SEPLLM_CUDA_ERROR;
-    g_static_ptr[dev] = static_cast<int32_t*>(p);
-  }
-  *out = g_static_ptr[dev];
+  void* p = nullptr;
+  SEPLLM_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_chunk_sums));
+  if (!p) return SEPLLM_CUDA_ERROR;
+  *out = static_cast<int32_t*>(p);
   return SEPLLM_OK;
 }
 

@@ -9,15 +9,17 @@ import numpy as np
 sys.path.insert(0, os.path.join(os.path.dirname(__file__), "..", ".."))
 from oracle import sepllm_oracle as orc  # noqa: E402
 
-# ten tokens, separators at positions 3 and 7 (a comma and a full stop in a short sentence)
-FLAGS = np.array([0, 0, 0, 1, 0, 0, 0, 1, 0, 0], dtype=bool)
+# The ten-token input of the paper's mask figure caption, "ABC,DE.FG\n": the comma, the full stop
+# and the newline (positions 3, 6, 9) are separators.
+TEXT = "ABC,DE.FG\n"
+FLAGS = np.array([ch in ",.\n" for ch in TEXT], dtype=bool)
 A, N = 1, 2
 
 if __name__ == "__main__":
     M = orc.mask_matrix(FLAGS, A, N)
     out = os.path.join(os.path.dirname(__file__), "mask_10_tokens.txt")
     with open(out, "w") as f:
-        f.write("# Eq. 2 for 10 tokens, separators at 3 and 7, n_init = 1, n_neighbor = 2; rows = queries\n")
+        f.write("# Eq. 2 for the caption input ABC,DE.FG\\n (separators at 3, 6, 9), n_init = 1, n_neighbor = 2; rows = queries\n")
         for row in M:
             f.write("".join("1" if x else "." for x in row) + "\n")
     print(open(out).read())

@@ -18,7 +18,9 @@ def _run(B, Hq, Hkv, L, d, a, n, rho, seed, sep_ids=inputs.SEP_IDS, structure="i
     O, LSE = attn_fwd(Q.cuda(), K.cuda(), V.cuda(), idesc, index)
     Oref, LSEref = orc.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(),
                                 flags_of(ids, sep_ids), a, n)
-    assert_close(O.float().cpu().numpy(), Oref, TOL_O, "O")
+    # n = 1 or 2: rows that keep one or two keys copy V rows, whose entries reach 4 and more, where
+    # a bf16 output is 0.016 off by rounding alone; only there is the bound taken relative
+    assert_close(O.float().cpu().numpy(), Oref, TOL_O, "O", scaled=(n <= 2))
     assert np.abs(LSE.cpu().numpy() - LSEref).max() <= TOL_LSE
     return O, LSE
 

@@ -25,7 +25,8 @@ def _compare(ids, sep_ids, a, n, BM=128, BN=128, side_cap=None, slow=False):
     return got
 
 
-@pytest.mark.parametrize("name", ["tiny", "pythia160m", "llama8b_prefill", "llama8b_long_r10", "llama8b_long_r20"])
+@pytest.mark.parametrize("name", ["tiny", "pythia160m", "llama8b_prefill", "llama8b_long_r05", "llama8b_long_r10",
+                                  "llama8b_long_r20"])
 def test_index_matches_oracle_on_workloads(name):
     c = inputs.CONFIGS[name]
     ids = inputs.token_ids(c["seed"], c["B"], c["L"], c["rho"], c["structure"])

@@ -5,7 +5,8 @@ import pytest
 
 from oracle import sepllm_oracle as orc
 from paper_2412_12094_b200 import api, inputs
-from tests._gpu_util import TOL_GRAD, TOL_LSE, TOL_O, assert_close, attn_bwd, attn_fwd, build_index, errors, flags_of
+from tests._gpu_util import (TOL_GRAD, TOL_LSE, TOL_O, assert_close, assert_grad_close, attn_bwd, attn_fwd,
+                             build_index, errors, flags_of)
 
 pytestmark = pytest.mark.gpu
 
@@ -38,20 +39,21 @@ def test_random_shape(seed):
     Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
     O, LSE = attn_fwd(Qd, Kd, Vd, idesc, index)
     Oref, LSEref = orc.attn_fwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), f, a, n)
-    assert_close(O.float().cpu().numpy(), Oref, TOL_O, f"O {c}")
+    # n = 1 or 2: rows that keep one or two keys copy V rows, whose entries reach 4 and more, where
+    # a bf16 output is 0.016 off by rounding alone; only there is the bound taken relative
+    assert_close(O.float().cpu().numpy(), Oref, TOL_O, f"O {c}", scaled=(n <= 2))
     assert np.abs(LSE.cpu().numpy() - LSEref).max() <= TOL_LSE, c
     grads = attn_bwd(dOd, Qd, Kd, Vd, O, LSE, idesc, index, grad_dtype=c["gd"])
-    refs = orc.attn_bwd(Q.double().numpy(), K.double().numpy(), V.double().numpy(), dO.double().numpy(), f, a, n)
-    for got_g, ref_g, what in zip(grads, refs, ("dQ", "dK", "dV")):
+    Qn, Kn, Vn, dOn = (t.double().numpy() for t in (Q, K, V, dO))
+    refs = orc.attn_bwd(Qn, Kn, Vn, dOn, f, a, n)
+    scales = orc.attn_bwd_term_scale(Qn, Kn, Vn, dOn, f, a, n)
+    for got_g, ref_g, rss, what in zip(grads, refs, scales, ("dQ", "dK", "dV")):
         got_g = got_g.float().cpu().numpy()
-        # Where a handful of keys collect thousands of weights near 1/8 (n = 1 or 2, no side entries)
-        # gradient entries reach 10 and more and the bf16 rounding of dS, 2^-9 of each term, adds up
-        # in proportion: the absolute bound is taken relative to the tensor's largest entry there.
-        big = max(1.0, float(np.abs(ref_g).max()))
-        diff = np.abs(got_g - ref_g)
-        assert np.isfinite(got_g).all(), (what, c)
-        assert diff.max() <= TOL_GRAD["max_abs"] * big, (what, float(diff.max()), big, c)
+        # Plain absolute bound, except for entries whose own terms are large enough for the bf16
+        # rounding of P / dS to exceed it: where a handful of keys collect thousands of weights
+        # (tiny n, hardly any side entries, or a wide query group) single entries reach 10 and more.
+        assert_grad_close(got_g, ref_g, rss, f"{what} {c}", bf16_out=(c["gd"] == 0))
         if np.linalg.norm(ref_g) > 1e-6:      # n = 1 without side entries: every dQ and dK is exactly 0
             assert errors(got_g, ref_g)[1] <= TOL_GRAD["rel_fro"], (what, errors(got_g, ref_g), c)
         else:
-            assert diff.max() <= 1e-4, (what, float(diff.max()), c)
+            assert np.abs(got_g - ref_g).max() <= 1e-4, (what, c)

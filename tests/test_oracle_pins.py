@@ -43,18 +43,22 @@ def test_mask_matches_set_construction(a, n):
         assert set(np.nonzero(M[i])[0].tolist()) == _kept_set_from_words(f, a, n, i)
     rows = np.array([0, 5, 50, 95])
     assert (orc.mask_rows(f, a, n, rows) == M[rows]).all()
+    cols = np.array([0, 1, 4, 49, 50, 51, 94, 95])
+    assert (orc.mask_rows(f, a, n, rows, cols) == M[np.ix_(rows, cols)]).all()
 
 
 def test_mask_regression_golden_ten_tokens():
-    """Not a value of the paper (its mask figure is an image): the ten-token mask as written out
-    by tests/golden/make_mask_golden.py, read back and checked by hand against Section 3.1 (row 9
-    keeps token 0, the separators 3 and 7, and tokens 8, 9)."""
+    """Not a value of the paper (its mask figure is an image, only the caption's input "ABC,DE.FG\\n"
+    is text): the mask of that input as written out by tests/golden/make_mask_golden.py, read back
+    and checked by hand against Section 3.1 (row 9, the newline, keeps token 0, the separators 3
+    and 6, and tokens 8, 9; row 7 keeps 0, 3 and the window 6, 7)."""
     sys_path = os.path.join(GOLD, "mask_10_tokens.txt")
     rows = [l.strip() for l in open(sys_path) if l.strip() and not l.startswith("#")]
-    f = np.array([0, 0, 0, 1, 0, 0, 0, 1, 0, 0], dtype=bool)
+    f = np.array([ch in ",.\n" for ch in "ABC,DE.FG\n"], dtype=bool)
+    assert np.flatnonzero(f).tolist() == [3, 6, 9]
     M = orc.mask_matrix(f, 1, 2)
     assert ["".join("1" if x else "." for x in r) for r in M] == rows
-    assert rows[9] == "1..1...111" and rows[4] == "1..11....." and rows[0] == "1........."
+    assert rows[9] == "1..1..1.11" and rows[7] == "1..1..11.." and rows[4] == "1..11....." and rows[0] == "1........."
 
 
 def test_fixed_interval_variant_mask():
@@ -374,6 +378,75 @@ def test_selected_key_gradients_equal_the_all_rows_backward():
     gk, gv = orc.attn_keys_bwd(Q, K, V, dO, f, a, n, keys)
     assert np.allclose(gk, dK[keys], rtol=1e-12, atol=1e-12)
     assert np.allclose(gv, dV[keys], rtol=1e-12, atol=1e-12)
+
+
+def test_blocked_key_gradients_equal_the_all_rows_backward():
+    """attn_keys_bwd_blocked (keys that nearly every row keeps, rows taken in blocks, columns no
+    row of a block keeps left out) against attn_bwd_head; block sizes that split the rows
+    unevenly, keys of every class (initial token, separators, plain tokens near and far)."""
+    rng = np.random.default_rng(6)
+    L, d, a, n = 150, 8, 2, 9
+    f = rng.random(L) < 0.15
+    Q, K, V, dO = (rng.standard_normal((L, d)) for _ in range(4))
+    M = orc.mask_matrix(f, a, n)
+    _, dK, dV = orc.attn_bwd_head(Q, K, V, dO, M)
+    seps = np.flatnonzero(f)
+    keys = np.unique(np.concatenate([[0, 1, 2, 60, 149], seps[:3], seps[-2:]]))
+    for block in (7, 64, 1000):
+        gk, gv = orc.attn_keys_bwd_blocked(Q, K, V, dO, f, a, n, keys, block_rows=block)
+        assert np.allclose(gk, dK[keys], rtol=1e-12, atol=1e-12)
+        assert np.allclose(gv, dV[keys], rtol=1e-12, atol=1e-12)
+    # the squared term sizes of the same keys against the all-rows version
+    flags2 = f[None, :]
+    _, sK, sV = orc.attn_bwd_term_scale(Q[None, None], K[None, None], V[None, None], dO[None, None], flags2, a, n)
+    _, _, k2, v2 = orc.attn_keys_bwd_blocked(Q, K, V, dO, f, a, n, keys, block_rows=13, with_term_scale=True)
+    assert np.allclose(np.sqrt(k2), sK[0, 0][keys], rtol=1e-10) and np.allclose(np.sqrt(v2), sV[0, 0][keys], rtol=1e-10)
+    # unsorted key list, custom scale
+    perm = keys[::-1]
+    gk, gv = orc.attn_keys_bwd_blocked(Q, K, V, dO, f, a, n, perm, scale=0.3, block_rows=11)
+    _, dK3, dV3 = orc.attn_bwd_head(Q, K, V, dO, M, 0.3)
+    assert np.allclose(gk, dK3[perm], atol=1e-12) and np.allclose(gv, dV3[perm], atol=1e-12)
+
+
+def test_term_scale_is_the_root_sum_square_of_the_gradient_terms():
+    """attn_bwd_term_scale against the terms written out one by one with torch (softmax over an
+    explicitly built kept set), including the sum over the query heads of a group; and the two
+    inequalities any root-sum-square obeys against the gradient itself."""
+    rng = np.random.default_rng(8)
+    B, Hq, Hkv, L, d, a, n = 1, 4, 2, 40, 4, 1, 5
+    G = Hq // Hkv
+    f = rng.random((B, L)) < 0.2
+    Q = rng.standard_normal((B, Hq, L, d))
+    K = rng.standard_normal((B, Hkv, L, d))
+    V = rng.standard_normal((B, Hkv, L, d))
+    dO = rng.standard_normal((B, Hq, L, d))
+    sQ, sK, sV = orc.attn_bwd_term_scale(Q, K, V, dO, f, a, n)
+    keep = torch.zeros((L, L), dtype=torch.bool)
+    for i in range(L):
+        keep[i, sorted(_kept_set_from_words(f[0], a, n, i))] = True
+    tK = torch.zeros((Hkv, L, d), dtype=torch.float64)
+    tV = torch.zeros((Hkv, L, d), dtype=torch.float64)
+    for h in range(Hq):
+        q, k, v, g = (torch.from_numpy(x) for x in (Q[0, h], K[0, h // G], V[0, h // G], dO[0, h]))
+        lam = (q @ k.T) / math.sqrt(d)
+        A = torch.softmax(lam.masked_fill(~keep, float("-inf")), dim=1)
+        o = A @ v
+        dlam = A * (g @ v.T - (g * o).sum(dim=1, keepdim=True))
+        s_row = ((g * o) ** 2).sum(dim=1).sqrt()                       # size of the products behind rowsum(dO * O)
+        terms_v = A[:, :, None] * g[:, None, :]                       # [i][j][e]
+        terms_k = dlam[:, :, None] * q[:, None, :] / math.sqrt(d)
+        terms_q = dlam[:, :, None] * k[None, :, :] / math.sqrt(d)     # [i][j][e]
+        extra_k = (A * s_row[:, None])[:, :, None] * q[:, None, :] / math.sqrt(d)
+        extra_q = (A * s_row[:, None])[:, :, None] * k[None, :, :] / math.sqrt(d)
+        tV[h // G] += (terms_v ** 2).sum(dim=0)
+        tK[h // G] += (terms_k ** 2).sum(dim=0) + (extra_k ** 2).sum(dim=0)
+        assert np.allclose(sQ[0, h], ((terms_q ** 2).sum(dim=1) + (extra_q ** 2).sum(dim=1)).sqrt().numpy(),
+                           rtol=1e-10, atol=1e-14)
+    assert np.allclose(sK[0], tK.sqrt().numpy(), rtol=1e-10, atol=1e-14)
+    assert np.allclose(sV[0], tV.sqrt().numpy(), rtol=1e-10, atol=1e-14)
+    dQ, dK, dV = orc.attn_bwd(Q, K, V, dO, f, a, n)
+    for grad, s, terms in ((dQ, sQ, L), (dK, sK, L * G), (dV, sV, L * G)):
+        assert (np.abs(grad) <= math.sqrt(terms) * s + 1e-12).all()      # Cauchy-Schwarz
 
 
 def test_rope_decode_pins():

@@ -87,9 +87,23 @@ typedef struct {
 
 /* Streaming cache capacities in the paper's names (Section 3.3): a initial,
  * s separator, w local window, c total; a + s + w < c, w >= 1.  The cache
- * calls take up to 16 query heads per kv head (Hq / Hkv <= 16). */
+ * calls take up to 16 query heads per kv head (Hq / Hkv <= 16).
+ * flags = 0: the four-block cache of Section 3.3 (the neighbour run grows until
+ *   Size_run reaches c, then its Past Window part is compacted).
+ * flags = SEPLLM_CACHE_FIXED_WINDOW: generation in the fundamental design
+ *   (Section 3.2 "Generation"; Section 4.2 keeps all separator KV there): the
+ *   neighbour run is exactly the w most recent tokens (w plays n's role); a
+ *   token that leaves it moves to the Separator Cache if it is a separator and
+ *   is dropped otherwise; the Separator Cache never evicts.  s is then its
+ *   capacity, chosen by the caller for the longest text (c only sizes the
+ *   buffers: slots = c + s as before, a + s + w < c).  After token t the
+ *   retained set is row t of Eq. 2's mask with n_init = a, n_neighbor = w.  A
+ *   sequence with more than s separators outside the window reports
+ *   SEPLLM_CAPACITY_EXCEEDED in the state's status word and keeps the newest s. */
+#define SEPLLM_CACHE_FIXED_WINDOW 1
 typedef struct {
   int32_t B, Hkv, Hq, d, a, s, w, c;
+  int32_t flags;
 } sepllm_cache_desc;
 
 /* ---- index blob -----------------------------------------------------------
@@ -216,7 +230,7 @@ typedef struct {
   int32_t slots;                 /* c + s */
   sepllm_cache_desc desc;
   int64_t off_seq, off_slot_pos, off_slot_is_sep, total_bytes;
-  int64_t reserved[22];
+  int64_t reserved[21];
 } sepllm_cache_header; /* 256 bytes */
 
 /* Per-sequence record inside the state, 16 int32.  reserved[0] is a scratch

@@ -515,6 +515,48 @@ class StreamingCache:
         return self.init + self.sep + self.window
 
 
+class FundamentalCache:
+    """Generation in the fundamental design (Section 3.2, "Generation"): after every token the KV
+    kept are those of the initial tokens, of every separator seen so far and of the ``n`` most
+    recent tokens; Section 4.2 runs this setting with all separator KV kept.  There is no
+    capacity and nothing is ever evicted from the separator list.  A token that falls out of the
+    window of the ``n`` most recent ones is kept on if it is a separator and dropped otherwise.
+    Same attribute names as :class:`StreamingCache` (``compactions`` counts the steps at which a
+    token left the window)."""
+
+    def __init__(self, a: int, n: int):
+        if n < 1:
+            raise ValueError("n >= 1: the current token always attends to itself")
+        self.a, self.n = a, n
+        self.init: List[int] = []
+        self.sep: List[int] = []
+        self.window: List[int] = []
+        self.window_is_sep: List[bool] = []
+        self.next_pos = 0
+        self.compactions = 0
+
+    @property
+    def size_run(self):
+        return len(self.init) + len(self.sep) + len(self.window)
+
+    def update(self, is_sep: bool) -> None:
+        pos = self.next_pos
+        self.next_pos += 1
+        if len(self.init) < self.a:
+            self.init.append(pos)
+            return
+        self.window.append(pos)
+        self.window_is_sep.append(bool(is_sep))
+        if len(self.window) > self.n:
+            left, was_sep = self.window.pop(0), self.window_is_sep.pop(0)
+            if was_sep:
+                self.sep.append(left)
+            self.compactions += 1
+
+    def retained(self) -> List[int]:
+        return self.init + self.sep + self.window
+
+
 def cache_after_prompt(flags: Sequence[bool], a: int, s: int, w: int, c: int) -> StreamingCache:
     """The cache a prompt leaves behind for generation (Section 3.2 "Generation",
     Section 3.3): the state the machine above reaches after taking in the

@@ -42,8 +42,11 @@ class AttnDesc(C.Structure):
         self.n_events = len(events)
 
 
+CACHE_FIXED_WINDOW = 1
+
+
 class CacheDesc(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("B", "Hkv", "Hq", "d", "a", "s", "w", "c")]
+    _fields_ = [(n, C.c_int32) for n in ("B", "Hkv", "Hq", "d", "a", "s", "w", "c", "flags")]
 
 
 class IndexHeader(C.Structure):
@@ -58,7 +61,7 @@ class CacheHeader(C.Structure):
     _fields_ = [("status", C.c_int32), ("magic", C.c_uint32), ("version", C.c_uint32),
                 ("slots", C.c_int32), ("desc", CacheDesc),
                 ("off_seq", C.c_int64), ("off_slot_pos", C.c_int64), ("off_slot_is_sep", C.c_int64),
-                ("total_bytes", C.c_int64), ("reserved", C.c_int64 * 22)]
+                ("total_bytes", C.c_int64), ("reserved", C.c_int64 * 21)]
 
 
 EXPORTS = [

@@ -35,6 +35,16 @@ __device__ __forceinline__ bool slot_active(const SlotGeom& g, int ns, int wlo, 
   return w >= g.wlo && w < g.whi;
 }
 
+struct FwdParams {
+  const int32_t* lim;        // [B][L]
+  const int32_t* tile_meta;  // [B][T][8]
+  __nv_bfloat16* O;
+  float* LSE;
+  int32_t* status;
+  int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap, pair_heads;
+  float scale_log2;
+};
+
 struct AttnLayout {
   int cap_pad;  // side_cap rounded up to 128 rows
   // forward workspace: status | Kside | Vside
@@ -56,6 +66,12 @@ __global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
                                const int32_t* __restrict__ n_side, int L, int Hkv, int side_cap,
                                int cap_pad, __nv_bfloat16* __restrict__ Ks,
                                __nv_bfloat16* __restrict__ Vs);
+
+// Forward for groups of four query heads at head size 128: two CTAs of a cluster work on the four
+// heads of one query tile as one MMA pair (attn_fwd_pair.cu).  Ks64 / K64: maps with 64-row boxes.
+sepllm_status launch_fwd_pair(const sepllm_attn_desc* d, const FwdParams& p, int n_tiles,
+                              const CUtensorMap& mq, const CUtensorMap& mk64, const CUtensorMap& mv,
+                              const CUtensorMap& mks64, const CUtensorMap& mvs, cudaStream_t stream);
 
 // Number of SMs of the current device (persistent kernels launch one CTA per SM).
 inline int sm_count() {

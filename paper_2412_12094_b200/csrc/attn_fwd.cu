@@ -108,16 +108,6 @@ struct FwdCfg {
 
 constexpr int kFwdThreads = 384;
 
-struct FwdParams {
-  const int32_t* lim;        // [B][L]
-  const int32_t* tile_meta;  // [B][T][8]
-  __nv_bfloat16* O;
-  float* LSE;
-  int32_t* status;
-  int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap, pair_heads;
-  float scale_log2;
-};
-
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
@@ -543,6 +533,16 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.pair_heads = (G % 2 == 0) ? 1 : 0;
   const float scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
   p.scale_log2 = scale * 1.4426950408889634f;
+  if (D == 128 && G % 4 == 0) {
+    // groups of four query heads: the CTA-pair kernel (K tiles loaded in 64-row halves)
+    CUtensorMap mk64, mks64;
+    if ((st = make_tile_map(&mk64, K, D, L, int64_t(d->B) * d->Hkv, D, L * D, 64)) != SEPLLM_OK) return st;
+    if ((st = make_tile_map(&mks64, Ks, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
+                            int64_t(lay.cap_pad) * D, 64)) != SEPLLM_OK) return st;
+    st = launch_fwd_pair(d, p, ih.n_tiles, mq, mk64, mv, mks64, mvs, stream);
+    record_event(d, 2, stream);
+    return st;
+  }
   const uint32_t smem = FwdCfg<D>::kRequest;
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_kernel<D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));

@@ -38,6 +38,7 @@ static sepllm_status fill_cache_header(const sepllm_cache_desc* d, sepllm_cache_
   if (d->Hq % d->Hkv != 0) return SEPLLM_INVALID_ARG;
   if (d->d != 64 && d->d != 128) return SEPLLM_UNSUPPORTED;
   if (d->Hq / d->Hkv > 16) return SEPLLM_UNSUPPORTED;
+  if (d->flags & ~SEPLLM_CACHE_FIXED_WINDOW) return SEPLLM_INVALID_ARG;
   *h = sepllm_cache_header{};
   h->magic = SEPLLM_CACHE_MAGIC;
   h->version = 1;
@@ -75,7 +76,13 @@ __device__ __forceinline__ UpdatePlan plan_update(const sepllm_cache_seq& q,
   const int ring = d.c - d.a;
   p.append_slot = d.a + d.s + (q.win_start + q.size_win) % ring;
   const int size_win = q.size_win + 1;
-  if (q.size_init + q.size_sep + size_win == d.c) {
+  if (d.flags & SEPLLM_CACHE_FIXED_WINDOW) {
+    // fundamental design: the run is the w most recent tokens; what is older leaves at once
+    if (size_win > d.w) {
+      p.compact = true;
+      p.n_past = size_win - d.w;
+    }
+  } else if (q.size_init + q.size_sep + size_win == d.c) {
     p.compact = true;
     p.n_past = size_win - d.w;
   }
@@ -264,6 +271,8 @@ cache_update(sepllm_cache_header h, uint8_t* __restrict__ state, __nv_bfloat16* 
   if (tid == 0) {
     pos_b[p.append_slot] = q.next_pos;
     sep_b[p.append_slot] = uint8_t(is_separator(new_token_ids[b], sep));
+    // a Separator Cache that is not meant to evict did
+    if ((d.flags & SEPLLM_CACHE_FIXED_WINDOW) && drop > 0) set_status(&v.hdr->status, SEPLLM_CAPACITY_EXCEEDED);
   }
   if (moves) {
     for (int k = tid; k < p.n_past; k += kUpdThreads) {
@@ -325,7 +334,15 @@ prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* _
     p.size_sep = 0;
     p.lo = d.a;
     p.compactions = 0;
-    if (T > d.a) {
+    bool overflow = false;
+    if (T > d.a && (d.flags & SEPLLM_CACHE_FIXED_WINDOW)) {
+      // fundamental design: the run is the last w tokens, every separator before it is kept
+      p.lo = max(d.a, T - d.w);
+      const int n_sep = cnt[p.lo] - cnt[d.a];
+      p.size_sep = min(d.s, n_sep);
+      overflow = d.s > 0 && n_sep > d.s;
+      p.compactions = p.lo - d.a;
+    } else if (T > d.a) {
       const int period = d.c - d.a - d.s - d.w;
       for (;;) {
         const int64_t t_full = int64_t(d.c) - d.a - p.size_sep + p.lo;  // tokens seen when Size_run = c
@@ -353,6 +370,7 @@ prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* _
     q.next_pos = T;
     v.seq[b] = q;
     if (bad) atomicExch(&v.hdr->status, SEPLLM_INVALID_ARG);
+    else if (overflow) set_status(&v.hdr->status, SEPLLM_CAPACITY_EXCEEDED);
   }
   if (b == 0) {
     // header: everything but the status word, which a failing block may be writing
@@ -822,7 +840,7 @@ static sepllm_status update_impl(const sepllm_cache_desc* desc, void* state, voi
   if (!aligned(state, kAlign) || !aligned(Kc, 16) || !aligned(Vc, 16) || !aligned(k_new, 16) ||
       !aligned(v_new, 16))
     return SEPLLM_INVALID_ARG;
-  const int max_past = desc->c - desc->a - desc->w;
+  const int max_past = (desc->flags & SEPLLM_CACHE_FIXED_WINDOW) ? 1 : desc->c - desc->a - desc->w;
   if (max_past > kMaxPast || desc->Hkv > 65535) return SEPLLM_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   SepIds sep;

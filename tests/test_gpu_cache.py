@@ -11,8 +11,8 @@ pytestmark = pytest.mark.gpu
 
 
 class GpuCache:
-    def __init__(self, B, Hkv, Hq, d, a, s, w, c):
-        self.desc = api.CacheDesc(B, Hkv, Hq, d, a, s, w, c)
+    def __init__(self, B, Hkv, Hq, d, a, s, w, c, flags=0):
+        self.desc = api.CacheDesc(B, Hkv, Hq, d, a, s, w, c, flags)
         sb, kb = api.sepllm_cache_bytes(self.desc)
         self.state = api.alloc_bytes(sb)
         self.Kc = torch.zeros(kb // 2, dtype=torch.bfloat16, device="cuda")

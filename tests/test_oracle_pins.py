@@ -319,6 +319,24 @@ def test_cache_after_prompt_has_the_content_the_blocks_are_defined_by():
 
 
 # ---------------------------------------------------------------- decode
+def test_fundamental_cache_retains_exactly_the_mask_row():
+    """Section 3.2: in generation the KV kept after token t are those row t of the mask keeps.
+    FundamentalCache against mask_matrix (pinned above to the section's wording) after every
+    token, for windows shorter and longer than the stream, with and without initial tokens."""
+    rng = np.random.default_rng(12)
+    for a, n, p in [(0, 1, 0.3), (2, 3, 0.3), (4, 9, 0.1), (3, 200, 0.2), (5, 4, 0.0), (1, 2, 1.0)]:
+        L = 70
+        f = rng.random(L) < p
+        M = orc.mask_matrix(f, a, n)
+        cache = orc.FundamentalCache(a, n)
+        for t in range(L):
+            cache.update(bool(f[t]))
+            assert sorted(cache.retained()) == np.flatnonzero(M[t]).tolist(), (a, n, t)
+            assert cache.retained() == sorted(cache.retained())          # position order
+            assert len(cache.window) == min(n, max(0, t + 1 - a))
+        assert cache.compactions == max(0, L - a - n)
+
+
 def test_decode_equals_last_prefill_row():
     L, d, a, n = 70, 8, 2, 9
     f, Q, K, V, _ = _rand_case(9, L, d, 0.2)

@@ -617,23 +617,34 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           tc_fence_after();
           issue_st(sq1);
         }
+        // the next dO tile is waited for here, off the chain that starts with P^T / dS^T below
+        if (it + 1 < n_it) wait(bar_of + (so ^ 1), opar1);
         wait(bar_pds, ipar);
         tc_fence_after();
         // Within the dP^T range, warpgroup u's columns [64u, 64u+64) hold P^T of its 64 queries
-        // in the first 32 and dS^T in the last 32.
+        // in the first 32 and dS^T in the last 32.  The three groups go to the pipe back to back:
+        // every gap in which the pipe runs dry costs a few hundred cycles of start-up on the
+        // chain dS^T(it) -> dV, dK, dP^T(it+1) -> dS^T(it+1), so the commits come after them.
         const uint32_t dot_lo = dot_lo0 + so * (C::kTile >> 4);
         const uint32_t qt_lo = qt_lo0 + sq * (C::kTile >> 4);
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k)
           umma_ts_lo(tmem + C::kdV, tmem + C::kdPT + (k >> 2) * 64 + (k & 3) * 8,
                      dot_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
-        tc_commit(bar_oe + so);
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k)
           umma_ts_lo(tmem + C::kdK, tmem + C::kdPT + (k >> 2) * 64 + 32 + (k & 3) * 8,
                      qt_lo + mnmajor_step(k), idesc_acc, (it > 0 || k > 0));
+        if (it + 1 < n_it) {
+          const uint32_t do_lo = do_lo0 + (so ^ 1) * (C::kTile >> 4);
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k)
+            umma_ss_lo(tmem + C::kdPT, v_lo + kmajor_step(k, kTileBlockBytes),
+                       do_lo + kmajor_step(k, kTileBlockBytes), idesc_s, k > 0);
+          tc_commit(bar_dpt);
+        }
+        tc_commit(bar_oe + so);
         tc_commit(bar_qe + sq);
-        if (it + 1 < n_it) issue_dpt(so ^ 1, opar1);
         sq = sq1;
         qpar = qpar1;
       }

@@ -544,7 +544,8 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
              const uint8_t* __restrict__ state, const __nv_bfloat16* __restrict__ Kc,
              const __nv_bfloat16* __restrict__ Vc, float* __restrict__ part_ml,
-             float* __restrict__ part_acc, int splits, const float2* __restrict__ rope) {
+             float* __restrict__ part_acc, int splits, const float2* __restrict__ rope,
+             int32_t* __restrict__ status) {
   constexpr int CH = D / 8;                 // 16-byte chunks per row
   constexpr int ROWB = D * 2;               // bytes per row
   constexpr int TILEB = kDecTile * ROWB;    // bytes of one K (or V) tile
@@ -557,6 +558,7 @@ decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __res
   const int G = d.Hq / d.Hkv;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0 && (split | hk | b) == 0) *status = SEPLLM_OK;
   CacheView cv = cache_view(const_cast<uint8_t*>(state), h);
   const sepllm_cache_seq sq = cv.seq[b];
   const int size_run = sq.size_init + sq.size_sep + sq.size_win;
@@ -935,7 +937,8 @@ extern "C" sepllm_status sepllm_decode_workspace_bytes(const sepllm_cache_desc* 
 template <int D, bool ROPE, bool WIDE>
 static sepllm_status launch_decode(const sepllm_cache_header& h, float scale_log2, const void* q,
                                    const void* state, const void* Kc, const void* Vc, float* ml,
-                                   float* acc, int splits, const float2* rope, cudaStream_t stream) {
+                                   float* acc, int splits, const float2* rope, int32_t* status,
+                                   cudaStream_t stream) {
   constexpr int smem = decode_smem_bytes<D>();
   static_assert(smem >= (kDecThreads / 32) * 16 * (8 + D * 4), "partials fit in the stage buffers");
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(decode_split<D, ROPE, WIDE>,
@@ -943,7 +946,7 @@ static sepllm_status launch_decode(const sepllm_cache_header& h, float scale_log
   decode_split<D, ROPE, WIDE><<<dim3(splits, h.desc.Hkv, h.desc.B), kDecThreads, smem, stream>>>(
       h, scale_log2, static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(state),
       static_cast<const __nv_bfloat16*>(Kc), static_cast<const __nv_bfloat16*>(Vc), ml, acc, splits,
-      rope);
+      rope, status);
   return SEPLLM_OK;
 }
 
@@ -951,12 +954,12 @@ template <int D>
 static sepllm_status dispatch_decode(bool with_rope, bool wide, const sepllm_cache_header& h,
                                      float scale_log2, const void* q, const void* state,
                                      const void* Kc, const void* Vc, float* ml, float* acc,
-                                     int splits, const float2* rope, cudaStream_t stream) {
-  if (with_rope)
-    return wide ? launch_decode<D, true, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
-                : launch_decode<D, true, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
-  return wide ? launch_decode<D, false, true>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
-              : launch_decode<D, false, false>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
+                                     int splits, const float2* rope, int32_t* status,
+                                     cudaStream_t stream) {
+#define SEPLLM_DEC(R, W) launch_decode<D, R, W>(h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, status, stream)
+  if (with_rope) return wide ? SEPLLM_DEC(true, true) : SEPLLM_DEC(true, false);
+  return wide ? SEPLLM_DEC(false, true) : SEPLLM_DEC(false, false);
+#undef SEPLLM_DEC
 }
 
 static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, const void* q,
@@ -975,16 +978,18 @@ static sepllm_status decode_impl(const sepllm_cache_desc* desc, float scale, con
   const int splits = decode_splits(desc);
   const size_t units = size_t(desc->B) * desc->Hq * splits;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  // the decode kernels have no bounded waits and report nothing: the status word reads OK
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(int32_t), stream));
+  // (the decode kernels have no bounded waits and report nothing: the split kernel writes the
+  // workspace's status word as OK itself, which saves a memset node per generated token)
   float* ml = reinterpret_cast<float*>(ws + kAlign);
   float* acc = reinterpret_cast<float*>(ws + kAlign + align_up(units * 2 * sizeof(float)));
   if (scale == 0.f) scale = 1.0f / sqrtf(float(desc->d));
   const float scale_log2 = scale * 1.4426950408889634f;
   const bool wide = desc->Hq / desc->Hkv > 8;
   st = (desc->d == 128)
-           ? dispatch_decode<128>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream)
-           : dispatch_decode<64>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope, stream);
+           ? dispatch_decode<128>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope,
+                                  reinterpret_cast<int32_t*>(ws), stream)
+           : dispatch_decode<64>(rope != nullptr, wide, h, scale_log2, q, state, Kc, Vc, ml, acc, splits, rope,
+                                 reinterpret_cast<int32_t*>(ws), stream);
   if (st != SEPLLM_OK) return st;
   if (desc->d == 128)
     decode_combine<128><<<dim3(desc->Hq, desc->B), 128, 0, stream>>>(

@@ -127,6 +127,12 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   };
   const int chunk = s_chunk;
   if (chunk >= n_chunks) return;
+  // Rows are divided by BM in several places; BM is a power of two in practice (128 for the
+  // attention calls), and a 64-bit division costs about a hundred instructions per thread.
+  const bool bm_pow2 = (BM & (BM - 1)) == 0;
+  const int bm_log2 = 31 - __clz(BM);
+  auto div_bm = [&](long long x) -> long long { return bm_pow2 ? (x >> bm_log2) : x / BM; };
+  auto mod_bm = [&](long long x) -> int { return bm_pow2 ? int(x & (BM - 1)) : int(x % BM); };
   const int32_t* ids = token_ids + static_cast<size_t>(b) * L;
   const int base = chunk * kIdxChunk;
 
@@ -182,25 +188,27 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   const long long row_lo = static_cast<long long>(base) + shift;
   const int n_rows = int(max(0LL, min(static_cast<long long>(L) - row_lo,
                                       static_cast<long long>(min(kIdxChunk, L - base)))));
-  const int t_first = int(row_lo / BM);
+  const int t_first = int(div_bm(row_lo));
   const bool fast_pairs = (BM >= kIdxPerThread) && (kIdxChunk / BM + 2 <= kMaxTilesPerChunk);
   for (int k = tid; k < kMaxTilesPerChunk; k += kIdxThreads) tile_part[k] = 0;
   __syncthreads();
   {
     int rel = warp_off + incl - local;
-    const int kb = BM - int((row_lo + p0) % BM);  // rows k >= kb belong to the next tile
+    const int kb = BM - mod_bm(row_lo + p0);  // rows k >= kb belong to the next tile
     int s0 = 0, s1 = 0;
+    // positions p0 .. p0+15 share p >> 5 (p0 is a multiple of 16): one base address, constant offsets
+    int32_t* mine = cnt_s + p0 + (p0 >> 5);
+    const int kv = n_rows - p0;   // rows k < kv exist
 #pragma unroll
     for (int k = 0; k < kIdxPerThread; ++k) {
-      const int p = p0 + k;
-      cnt_s[p + (p >> 5)] = rel;
-      const int vv = (p < n_rows) ? rel : 0;
+      mine[k] = rel;
+      const int vv = (k < kv) ? rel : 0;
       s0 += (k < kb) ? vv : 0;
       s1 += (k < kb) ? 0 : vv;
       rel += (fl >> k) & 1u;
     }
     if (fast_pairs) {
-      const int tl = int((row_lo + p0) / BM) - t_first;
+      const int tl = int(div_bm(row_lo + p0)) - t_first;
       if (s0) atomicAdd(&tile_part[tl], s0);
       if (s1) atomicAdd(&tile_part[tl + 1], s1);
     }
@@ -264,10 +272,11 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   if (base + kIdxChunk + shift <= L && base >= shift) {  // whole chunk inside both arrays
     int32_t* cdst = cnt_b + base + tid;
     int32_t* ldst = lim_b + base + shift + tid;
+    // position k * 256 + tid sits at word k * 264 + tid + wid of the padded buffer
+    const int32_t* src = cnt_s + tid + wid;
 #pragma unroll
     for (int k = 0; k < kIdxPerThread; ++k) {
-      const int p = k * kIdxThreads + tid;
-      const int v = cnt_s[p + (p >> 5)] + off;
+      const int v = src[k * (kIdxThreads + kIdxThreads / 32)] + off;
       cdst[k * kIdxThreads] = v;
       ldst[k * kIdxThreads] = v;
     }
@@ -301,7 +310,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   };
   if (n_rows > 0) {
     const long long row_hi = row_lo + n_rows;  // exclusive
-    const int t_last = int((row_hi - 1) / BM);
+    const int t_last = int(div_bm(row_hi - 1));
     for (int t = t_first + (fast_pairs ? tid : wid); t <= t_last; t += (fast_pairs ? kIdxThreads : kIdxThreads / 32)) {
       const long long r0 = max(row_lo, static_cast<long long>(t) * BM);
       const long long r1 = min(row_hi, (static_cast<long long>(t) + 1) * BM);
@@ -334,7 +343,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   }
   if (chunk == 0) {
     // tiles whose first row comes before row n_neighbor-1 belong to no chunk (lim is 0 there)
-    const int t_head = int(min(static_cast<long long>(T), (static_cast<long long>(shift) + BM - 1) / BM));
+    const int t_head = int(min(static_cast<long long>(T), div_bm(static_cast<long long>(shift) + BM - 1)));
     for (int t = tid; t < t_head; t += kIdxThreads) window_words(t);
     if (b == 0) {
       // header: everything but the status word, which any block may be setting

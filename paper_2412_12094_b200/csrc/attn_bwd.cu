@@ -545,7 +545,11 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
   };
   auto q_plane_of = [&](int it) { return b * p.Hq + hk * G + g_lo + it % n_g; };
-  auto q0_of = [&](int it) { return (t_lo + it / n_g) * kBM; };
+  // The side pass walks its query tiles from the end of the sequence backwards: the CTAs of
+  // neighbouring side tiles of one head, which start together, then read the same Q / dO tiles
+  // at the same time (one of them from DRAM, the others from L2) instead of each streaming the
+  // head's Q and dO at its own offset.
+  auto q0_of = [&](int it) { return (SIDE ? (t_hi - it / n_g) : (t_lo + it / n_g)) * kBM; };
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");

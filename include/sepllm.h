@@ -28,7 +28,12 @@
  *  - Sequences shorter than L are padded at the end (any token ids, any finite
  *    K, V, Q values): the mask is causal, so no valid row sees a padded key,
  *    and with dO = 0 on the padded rows the padded queries add nothing to dK
- *    and dV.  Outputs of padded rows are to be ignored.
+ *    and dV.  Outputs of padded rows are to be ignored.  An index built with
+ *    sepllm_build_index_varlen also tells the attention calls where each
+ *    sequence ends: query tiles that hold only padding are then skipped (their
+ *    rows of O, LSE and dQ are not written; their rows of dK and dV are
+ *    written as 0), and padded positions are never initial tokens or
+ *    separators.
  *  - Supported: d in {64, 128}; Hq a multiple of Hkv; n_neighbor >= 1;
  *    n_init >= 0; index tiles BM = BN = 128 for the attention calls.
  */
@@ -115,7 +120,9 @@ typedef struct {
  *   side_pos  [B][side_cap] ascending positions of side members (-1 beyond n_side)
  *   n_side    [B]           number of side members (may exceed side_cap: then the status
  *                           word reads SEPLLM_CAPACITY_EXCEEDED and side_pos is truncated)
- *   tile_meta [B][ceil(L/BM)][8] per query tile of BM rows:
+ *   seq_len   [B]           tokens in each sequence (L unless built by sepllm_build_index_varlen)
+ *   tile_meta [B][ceil(L/BM)][8] per query tile of BM rows (all 0 for a tile of padding; the last
+ *       valid tile ends at the sequence's last token):
  *       0 side_full   floor(lim[first row]/BN)   side tiles all rows see in full
  *       1 side_last   ceil(lim[last row]/BN)     side tiles any row sees
  *       2 win_lo      max(0, first row - n_neighbor + 1)
@@ -134,7 +141,8 @@ typedef struct {
   sepllm_index_desc desc;
   int32_t n_tiles;     /* ceil(L/BM) */
   int64_t off_cnt, off_lim, off_side_pos, off_n_side, off_tile_meta, total_bytes;
-  int64_t reserved[20];
+  int64_t off_seq_len;
+  int64_t reserved[19];
 } sepllm_index_header; /* 256 bytes */
 
 /* Sizes of the index blob and of the scratch buffer sepllm_build_index needs. */
@@ -151,6 +159,18 @@ sepllm_status sepllm_index_bytes(const sepllm_index_desc* desc, size_t* index_by
 sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* token_ids,
                                  const int32_t* sep_ids, void* index, void* scratch,
                                  void* stream);
+
+/* Index of a batch of sequences of unequal lengths padded to L (the paper
+ * trains and pre-fills on full rows and does not treat padding; the reading
+ * taken is that a padded position is no token at all): seq_len dev int32 [B],
+ * 0 <= seq_len[b] <= L (values outside are clamped).  Positions from
+ * seq_len[b] on are neither initial tokens nor separators, query tiles that
+ * start at or behind seq_len[b] carry no work, and the tile that holds the
+ * last token ends there.  With every seq_len[b] = L the result equals
+ * sepllm_build_index's.  Other arguments as there. */
+sepllm_status sepllm_build_index_varlen(const sepllm_index_desc* desc, const int32_t* token_ids,
+                                        const int32_t* seq_len, const int32_t* sep_ids,
+                                        void* index, void* scratch, void* stream);
 
 /* Same result as sepllm_build_index, for callers that cannot hand over a scratch
  * buffer because they cannot allocate device memory at the point of the call: a

@@ -353,8 +353,16 @@ def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None 
 # ----------------------------------------------------------------------------
 
 def build_index(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int,
-                side_cap: int):
+                side_cap: int, seq_len=None):
     """Canonical index arrays for a batch of sequences.
+
+    seq_len (optional, one length per sequence): sequence b holds seq_len[b]
+    tokens, the rest of its row is padding.  The paper does not treat batches
+    of unequal lengths; the reading taken here is the obvious one: a padded
+    position is no token (no initial token, no separator), a query tile whose
+    first row is padding has no work (all eight metadata words 0), the last
+    valid tile ends at the last valid row, and ``pairs`` counts valid rows only.
+    cnt and lim keep their formulas on every position of the row.
 
     side member g[j] = (j < a) or f[j]            (initial tokens and separators)
     cnt[j]  = number of side members at positions < j, j = 0..L
@@ -380,11 +388,13 @@ def build_index(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int
     n_side = np.zeros((B,), dtype=np.int32)
     tile_meta = np.zeros((B, T, 8), dtype=np.int32)
     sep = set(int(x) for x in sep_ids)
+    lens = np.full((B,), L, dtype=np.int32) if seq_len is None else np.asarray(seq_len, dtype=np.int32)
     for b in range(B):
+        Lv = int(lens[b])
         k = 0
         for j in range(L):
             cnt[b, j] = k
-            if j < a or int(token_ids[b, j]) in sep:
+            if j < Lv and (j < a or int(token_ids[b, j]) in sep):
                 if k < side_cap:
                     side_pos[b, k] = j
                 k += 1
@@ -394,7 +404,9 @@ def build_index(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int
             lim[b, i] = cnt[b, max(0, i - n + 1)]
         for t in range(T):
             r0 = t * BM
-            r1 = min(L, (t + 1) * BM) - 1
+            if r0 >= Lv:
+                continue                      # a tile of padding: all words stay 0
+            r1 = min(Lv, (t + 1) * BM) - 1
             pairs = 0
             for i in range(r0, r1 + 1):
                 pairs += int(lim[b, i]) + min(i + 1, n)
@@ -402,18 +414,20 @@ def build_index(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int
             win_hi = r1 + 1
             tile_meta[b, t] = [int(lim[b, r0]) // BN, -(-int(lim[b, r1]) // BN), win_lo, win_hi,
                                win_lo // BN, -(-win_hi // BN), pairs, 0]
-    return dict(cnt=cnt, lim=lim, side_pos=side_pos, n_side=n_side, tile_meta=tile_meta)
+    return dict(cnt=cnt, lim=lim, side_pos=side_pos, n_side=n_side, tile_meta=tile_meta, seq_len=lens)
 
 
 def build_index_fast(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN: int,
-                     side_cap: int):
+                     side_cap: int, seq_len=None):
     """Same arrays as :func:`build_index`, with numpy prefix sums in place of
     the Python loops, for sequences too long to loop over.  Tests check the two
     against each other."""
     token_ids = np.asarray(token_ids)
     B, L = token_ids.shape
     T = (L + BM - 1) // BM
+    lens = np.full((B,), L, dtype=np.int32) if seq_len is None else np.asarray(seq_len, dtype=np.int32)
     g = np.isin(token_ids, np.asarray(list(sep_ids))) | (np.arange(L)[None, :] < a)
+    g &= np.arange(L)[None, :] < lens[:, None]
     cnt = np.zeros((B, L + 1), dtype=np.int64)
     cnt[:, 1:] = np.cumsum(g, axis=1)
     i = np.arange(L)
@@ -424,20 +438,19 @@ def build_index_fast(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN
         side_pos[b, :p.size] = p
     per_row = lim + np.minimum(i + 1, n)[None, :]
     tile_meta = np.zeros((B, T, 8), dtype=np.int32)
-    for t in range(T):
-        r0 = t * BM
-        r1 = min(L, (t + 1) * BM) - 1
-        win_lo = max(0, r0 - n + 1)
-        win_hi = r1 + 1
-        tile_meta[:, t, 0] = lim[:, r0] // BN
-        tile_meta[:, t, 1] = -(-lim[:, r1] // BN)
-        tile_meta[:, t, 2] = win_lo
-        tile_meta[:, t, 3] = win_hi
-        tile_meta[:, t, 4] = win_lo // BN
-        tile_meta[:, t, 5] = -(-win_hi // BN)
-        tile_meta[:, t, 6] = per_row[:, r0:r1 + 1].sum(axis=1)
+    for b in range(B):
+        Lv = int(lens[b])
+        for t in range(T):
+            r0 = t * BM
+            if r0 >= Lv:
+                break
+            r1 = min(Lv, (t + 1) * BM) - 1
+            win_lo = max(0, r0 - n + 1)
+            win_hi = r1 + 1
+            tile_meta[b, t] = [lim[b, r0] // BN, -(-lim[b, r1] // BN), win_lo, win_hi, win_lo // BN,
+                               -(-win_hi // BN), per_row[b, r0:r1 + 1].sum(), 0]
     return dict(cnt=cnt.astype(np.int32), lim=lim.astype(np.int32), side_pos=side_pos,
-                n_side=cnt[:, L].astype(np.int32), tile_meta=tile_meta)
+                n_side=cnt[:, L].astype(np.int32), tile_meta=tile_meta, seq_len=lens)
 
 
 # ----------------------------------------------------------------------------

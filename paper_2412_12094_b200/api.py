@@ -54,7 +54,7 @@ class IndexHeader(C.Structure):
                 ("desc", IndexDesc), ("n_tiles", C.c_int32),
                 ("off_cnt", C.c_int64), ("off_lim", C.c_int64), ("off_side_pos", C.c_int64),
                 ("off_n_side", C.c_int64), ("off_tile_meta", C.c_int64), ("total_bytes", C.c_int64),
-                ("reserved", C.c_int64 * 20)]
+                ("off_seq_len", C.c_int64), ("reserved", C.c_int64 * 19)]
 
 
 class CacheHeader(C.Structure):
@@ -65,7 +65,7 @@ class CacheHeader(C.Structure):
 
 
 EXPORTS = [
-    "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_static",
+    "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_varlen", "sepllm_build_index_static",
     "sepllm_build_index_fixed_interval",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
@@ -142,6 +142,14 @@ def sepllm_build_index(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index:
                                     _stream()), "sepllm_build_index")
 
 
+def sepllm_build_index_varlen(desc: IndexDesc, token_ids: torch.Tensor, seq_len: torch.Tensor, sep_ids,
+                              index: torch.Tensor, scratch: torch.Tensor):
+    arr, p, n = _sep_array(sep_ids)
+    assert n == desc.n_sep
+    _check(lib().sepllm_build_index_varlen(C.byref(desc), _ptr(token_ids), _ptr(seq_len), p, _ptr(index),
+                                           _ptr(scratch), _stream()), "sepllm_build_index_varlen")
+
+
 def sepllm_build_index_static(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index: torch.Tensor):
     """Index build for callers that cannot allocate a scratch buffer: the library's own fixed
     array is used instead (B * (2 * ceil(L/4096) + 1) <= 65536).  Calls that may overlap on the GPU must be
@@ -176,6 +184,7 @@ def read_index(index: torch.Tensor) -> dict:
         side_pos=arr(h.off_side_pos, d.B * d.side_cap).reshape(d.B, d.side_cap),
         n_side=arr(h.off_n_side, d.B),
         tile_meta=arr(h.off_tile_meta, d.B * T * 8).reshape(d.B, T, 8),
+        seq_len=arr(h.off_seq_len, d.B),
     )
 
 

@@ -55,6 +55,7 @@ struct BwdParams {
   const int32_t* side_pos;   // [B][side_cap]
   const int32_t* n_side;     // [B]
   const int32_t* tile_meta;  // [B][T][8]
+  const int32_t* seq_len;    // [B]
   const float2* stats;       // [B][Hq][L] (LSE * log2 e, Delta)
   float* dKs;                // [split][B][Hkv][cap_pad][D] fp32 side partials
   float* dVs;
@@ -123,12 +124,12 @@ __device__ __forceinline__ DqItem dq_item(const BwdParams& p, int w) {
   it.b = x / p.Hq;
   const int hq = x % p.Hq;
   it.t = p.T - 1 - w / hb;
-  const SlotGeom g = load_slot(p.tile_meta, it.b, p.T, it.t, hq, p.cap_pad / kBN);
+  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, it.b, p.T, it.t, hq, p.cap_pad / kBN);
   it.kv_plane = it.b * p.Hkv + hq / (p.Hq / p.Hkv);
   it.q_plane = it.b * p.Hq + hq;
   it.ns = g.ns;
   it.wlo = g.wlo;
-  it.n_tiles = g.ns + (g.whi - g.wlo);
+  it.n_tiles = (g.t >= 0) ? g.ns + (g.whi - g.wlo) : 0;   // 0: a tile of padding, skipped by every role
   it.side_full = g.side_full;
   return it;
 }
@@ -200,7 +201,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       // ---------------- TMA producer ----------------
       int tb = 0;  // tiles before this item
       for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
-        const DqItem it = dq_item(p, w);
+        const DqItem it = dq_item(p, w);   // (an empty item has no tiles)
         for (int j = 0; j < it.n_tiles; ++j) {
           const bool side = j < it.ns;
           const int y = side ? j * kBN : (it.wlo + (j - it.ns)) * kBN;
@@ -247,8 +248,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       int st = 0;            // ring stage of the current tile
       uint32_t fpar = 0;     // parity of that stage's "full" barrier
       uint32_t gpar = 0;     // parity of the per-tile barriers (tile counter & 1)
-      for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++ino) {
+      for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
         const int n_tiles = dq_item(p, w).n_tiles;
+        if (n_tiles == 0) continue;
         wait(bar_qdo, ino & 1);
         wait(bar_f + st, fpar);
         tc_fence_after();
@@ -282,6 +284,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
           gpar ^= 1u;
         }
         tc_commit(bar_acc);
+        ++ino;
       }
     }
   } else {
@@ -313,9 +316,16 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       mbar_arrive_warp(bar_qdo);
     };
     int tb = 0, ino = 0;
-    if (int(blockIdx.x) < n_items) load_qdo(dq_item(p, blockIdx.x));
-    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++ino) {
+    // the next item of this CTA that has work, from w on
+    auto next_item = [&](int w) {
+      while (w < n_items && dq_item(p, w).n_tiles == 0) w += gridDim.x;
+      return w;
+    };
+    int w = next_item(blockIdx.x);
+    if (w < n_items) load_qdo(dq_item(p, w));
+    for (; w < n_items; ++ino) {
       const DqItem it = dq_item(p, w);
+      const int w_next = next_item(w + gridDim.x);
       const int t = it.t, ns = it.ns;
       const int row = t * kBM + r;
       const bool row_ok = row < p.L;
@@ -396,7 +406,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tb += it.n_tiles;
       // Every S and dP MMA of this item is complete (the last dP was waited for), so Q and dO of
       // the next item can go into tensor memory while this item's last dQ MMAs run.
-      if (w + int(gridDim.x) < n_items) load_qdo(dq_item(p, w + gridDim.x));
+      if (w_next < n_items) load_qdo(dq_item(p, w_next));
       // ---------------- epilogue: each warpgroup stores half of the row ----------------
       wait(bar_acc, ino & 1);
       tc_fence_after();
@@ -418,6 +428,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
                             p.grad_fp32, v);
         }
       }
+      w = w_next;
     }
   }
   tc_fence_before();
@@ -502,15 +513,17 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int kv_plane = b * p.Hkv + hk;
   const int ns = min(p.n_side[b], p.side_cap);
 
-  // query tiles [t_lo, t_hi] that keep at least one key of this tile
+  // query tiles [t_lo, t_hi] that keep at least one key of this tile; tiles of padding behind
+  // the sequence's last token (seq_len from the index) are left out
+  const int t_last = (p.seq_len[b] + kBM - 1) / kBM - 1;
   int t_lo, t_hi;
   if (SIDE) {
     if (kt * kBN >= ns) return;  // no entries in this side tile: nothing reads its partial rows
     t_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / kBM;
-    t_hi = p.T - 1;
+    t_hi = t_last;
   } else {
     t_lo = kt;  // kBM == kBN
-    t_hi = min(p.T - 1, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / kBM);
+    t_hi = min(t_last, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / kBM);
   }
   const int n_it = max(0, t_hi - t_lo + 1) * n_g;
 
@@ -810,8 +823,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t rr[32];
-        tmem_ld32(t_acc + c * 32, rr);
-        tmem_ld_wait();
+        if (n_it > 0) {
+          tmem_ld32(t_acc + c * 32, rr);
+          tmem_ld_wait();
+        } else {   // a key tile of padding: its rows of dK and dV are written as 0
+#pragma unroll
+          for (int e = 0; e < 32; ++e) rr[e] = 0;
+        }
         if (r_ok) {
           float v[32];
 #pragma unroll
@@ -879,6 +897,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.side_pos = side_pos;
   p.n_side = n_side;
   p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
+  p.seq_len = reinterpret_cast<const int32_t*>(index + ih.off_seq_len);
   p.stats = stats;
   p.dKs = reinterpret_cast<float*>(ws + lay.off_dks);
   p.dVs = reinterpret_cast<float*>(ws + lay.off_dvs);

@@ -12,12 +12,13 @@ constexpr uint32_t kTileBlockBytes = 128 * 128;  // 128 rows x 64 bf16, one swiz
 struct SlotGeom {
   int t, hq, side_full, ns, wlo, whi;
 };
-__device__ __forceinline__ SlotGeom load_slot(const int32_t* tile_meta, int b, int T, int t, int hq,
-                                              int side_tiles_cap) {
+// A tile that starts at or behind the end of its sequence (seq_len from the index) is empty too.
+__device__ __forceinline__ SlotGeom load_slot(const int32_t* tile_meta, const int32_t* seq_len, int b,
+                                              int T, int t, int hq, int side_tiles_cap) {
   SlotGeom g;
-  g.t = t;
+  g.t = (t >= 0 && t * kBM < seq_len[b]) ? t : -1;
   g.hq = hq;
-  if (t >= 0) {
+  if (g.t >= 0) {
     const int32_t* meta = tile_meta + (size_t(b) * T + t) * 8;
     g.side_full = meta[0];
     g.ns = min(meta[1], side_tiles_cap);
@@ -38,6 +39,7 @@ __device__ __forceinline__ bool slot_active(const SlotGeom& g, int ns, int wlo, 
 struct FwdParams {
   const int32_t* lim;        // [B][L]
   const int32_t* tile_meta;  // [B][T][8]
+  const int32_t* seq_len;    // [B]
   __nv_bfloat16* O;
   float* LSE;
   int32_t* status;

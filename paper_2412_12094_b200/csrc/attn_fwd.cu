@@ -141,17 +141,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   const int heads_x = p.pair_heads ? p.Hq / 2 : p.Hq;
   const int b = int(blockIdx.x) / heads_x, hx = int(blockIdx.x) % heads_x;
 
-  // the two slots of this CTA (slot 1 is never empty; slot 0 is when T is odd and tiles pair up)
+  // the two slots of this CTA (a slot is empty when its tile does not exist or holds only padding)
   SlotGeom g0, g1;
   if (p.pair_heads) {
     const int t = p.T - 1 - int(blockIdx.y);
-    g0 = load_slot(p.tile_meta, b, p.T, t, 2 * hx, p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, b, p.T, t, 2 * hx + 1, p.side_tiles_cap);
+    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx + 1, p.side_tiles_cap);
   } else {
     const int t = p.T - 1 - 2 * int(blockIdx.y);
-    g0 = load_slot(p.tile_meta, b, p.T, t - 1, hx, p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, b, p.T, t, hx, p.side_tiles_cap);
+    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t - 1, hx, p.side_tiles_cap);
+    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, hx, p.side_tiles_cap);
   }
+  if (g0.t < 0 && g1.t < 0) return;   // both tiles are padding: nothing to do, nothing written
   const int kv_plane = b * p.Hkv + g1.hq / G;
   // key tiles of the CTA: side tiles [0, ns), then window tiles [wlo, whi)
   const int ns = max(g0.ns, g1.ns);
@@ -519,6 +520,7 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   FwdParams p;
   p.lim = reinterpret_cast<const int32_t*>(index + ih.off_lim);
   p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
+  p.seq_len = reinterpret_cast<const int32_t*>(index + ih.off_seq_len);
   p.O = static_cast<__nv_bfloat16*>(O);
   p.LSE = LSE;
   p.status = reinterpret_cast<int32_t*>(ws);

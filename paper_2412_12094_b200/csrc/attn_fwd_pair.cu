@@ -90,7 +90,8 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
   const int b = int(blockIdx.x) / heads_x, hx = int(blockIdx.x) % heads_x;
   const int t = p.T - 1 - int(blockIdx.y);
   const int G = p.Hq / p.Hkv;
-  const SlotGeom g = load_slot(p.tile_meta, b, p.T, t, 2 * hx, p.side_tiles_cap);
+  if (t * kBM >= p.seq_len[b]) return;   // a tile of padding (the same for both CTAs of the pair)
+  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap);
   const int kv_plane = b * p.Hkv + (2 * hx) / G;
   const int ns = g.ns, wlo = g.wlo;
   const int n_tiles = ns + (g.whi - g.wlo);

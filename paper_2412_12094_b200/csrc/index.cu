@@ -105,7 +105,8 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
            int n_chunks, int side_cap, int32_t* __restrict__ cnt, int32_t* __restrict__ lim,
            int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
            int32_t* __restrict__ tile_meta, int T, int BM, int BN, int interval,
-           const __grid_constant__ sepllm_index_header hdr, int32_t* status) {
+           const __grid_constant__ sepllm_index_header hdr, int32_t* status,
+           const int32_t* __restrict__ seq_len, int32_t* __restrict__ seq_len_out) {
   __shared__ int warp_buf[kIdxThreads / 32];
   __shared__ int s_chunk, s_off;
   // counts of the chunk, one pad word per 32 so that a thread's 16 consecutive words and a
@@ -135,6 +136,8 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   auto mod_bm = [&](long long x) -> int { return bm_pow2 ? int(x & (BM - 1)) : int(x % BM); };
   const int32_t* ids = token_ids + static_cast<size_t>(b) * L;
   const int base = chunk * kIdxChunk;
+  // tokens in this sequence: positions from Lv on are padding (no members, no query rows)
+  const int Lv = seq_len ? max(0, min(L, seq_len[b])) : L;
 
   // flags of this thread's 16 consecutive positions
   const int p0 = tid * kIdxPerThread, j0 = base + p0;
@@ -161,6 +164,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
     const int m = max(0, min(kIdxPerThread, min(n_init, L) - j0));
     fl |= (1u << m) - 1u;
   }
+  if (j0 + kIdxPerThread > Lv) fl &= (j0 >= Lv) ? 0u : ((1u << (Lv - j0)) - 1u);   // padding holds no members
   const int local = __popc(fl);
 
   // exclusive scan of `local` over the block
@@ -186,7 +190,8 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   // lie in at most two query tiles, whose side-pair sums are gathered in shared memory.
   const int shift = n_neighbor - 1;
   const long long row_lo = static_cast<long long>(base) + shift;
-  const int n_rows = int(max(0LL, min(static_cast<long long>(L) - row_lo,
+  // (valid rows only: rows of padding count no pairs and belong to no tile with work)
+  const int n_rows = int(max(0LL, min(static_cast<long long>(Lv) - row_lo,
                                       static_cast<long long>(min(kIdxChunk, L - base)))));
   const int t_first = int(div_bm(row_lo));
   const bool fast_pairs = (BM >= kIdxPerThread) && (kIdxChunk / BM + 2 <= kMaxTilesPerChunk);
@@ -299,7 +304,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   // share of word 6) or last row (word 1).  tile_meta was zeroed before the launch.
   int32_t* meta_b = tile_meta + static_cast<size_t>(b) * T * 8;
   auto window_words = [&](int t) {
-    const int r0 = t * BM, r1 = min(L, (t + 1) * BM) - 1;
+    const int r0 = t * BM, r1 = min(Lv, (t + 1) * BM) - 1;
     const int win_lo = max(0, r0 - n_neighbor + 1), win_hi = r1 + 1;
     int32_t* m = meta_b + static_cast<size_t>(t) * 8;
     m[2] = win_lo;
@@ -328,7 +333,7 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
       if ((fast_pairs || lane == 0)) {
         if (sum) atomicAdd(&meta_b[size_t(t) * 8 + 6], sum);
         const long long first = static_cast<long long>(t) * BM;
-        const long long last = min(static_cast<long long>(L), first + BM) - 1;
+        const long long last = min(static_cast<long long>(Lv), first + BM) - 1;
         if (first >= row_lo) {  // this chunk holds the tile's first row
           const int p = int(first - row_lo);
           meta_b[size_t(t) * 8 + 0] = (cnt_s[p + (p >> 5)] + off) / BN;
@@ -343,8 +348,10 @@ index_scan(const int32_t* __restrict__ token_ids, int L, int n_init, int n_neigh
   }
   if (chunk == 0) {
     // tiles whose first row comes before row n_neighbor-1 belong to no chunk (lim is 0 there)
-    const int t_head = int(min(static_cast<long long>(T), div_bm(static_cast<long long>(shift) + BM - 1)));
+    const int Tv = int(div_bm(static_cast<long long>(Lv) + BM - 1));   // tiles that hold tokens
+    const int t_head = int(min(static_cast<long long>(Tv), div_bm(static_cast<long long>(shift) + BM - 1)));
     for (int t = tid; t < t_head; t += kIdxThreads) window_words(t);
+    if (tid == 0) seq_len_out[b] = Lv;
     if (b == 0) {
       // header: everything but the status word, which any block may be setting
       const int32_t* src = reinterpret_cast<const int32_t*>(&hdr);
@@ -398,6 +405,8 @@ sepllm_status fill_index_header(const sepllm_index_desc* d, sepllm_index_header*
   off = align_up(off + sizeof(int32_t) * size_t(d->B));
   h->off_tile_meta = off;
   off = align_up(off + sizeof(int32_t) * size_t(d->B) * h->n_tiles * 8);
+  h->off_seq_len = off;
+  off = align_up(off + sizeof(int32_t) * size_t(d->B));
   h->total_bytes = off;
   return SEPLLM_OK;
 }
@@ -411,7 +420,8 @@ static_assert(sizeof(sepllm_index_header) == 256, "index header is 256 bytes");
 // Launches shared by the two entry points.  `scratch` holds index_scratch_words() int32 words.
 static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_index_header& h,
                                   const int32_t* token_ids, const int32_t* sep_ids, uint8_t* blob,
-                                  int32_t* scratch, cudaStream_t stream, int interval = 0) {
+                                  int32_t* scratch, cudaStream_t stream, int interval = 0,
+                                  const int32_t* seq_len = nullptr) {
   SepIds sep;
   sep.n = desc->n_sep;
   for (int k = 0; k < SEPLLM_MAX_SEP_IDS; ++k)
@@ -434,7 +444,8 @@ static sepllm_status launch_index(const sepllm_index_desc* desc, const sepllm_in
       reinterpret_cast<int32_t*>(blob + h.off_side_pos),                                         \
       reinterpret_cast<int32_t*>(blob + h.off_n_side),                                           \
       reinterpret_cast<int32_t*>(blob + h.off_tile_meta), h.n_tiles, desc->BM, desc->BN,         \
-      interval, h, reinterpret_cast<int32_t*>(blob))
+      interval, h, reinterpret_cast<int32_t*>(blob), seq_len,                                    \
+      reinterpret_cast<int32_t*>(blob + h.off_seq_len))
   SepTable tab;
   tab.mult = 0;
   const bool hashed = sep.n > 0 && build_sep_table(sep_ids, sep.n, &tab);
@@ -474,6 +485,23 @@ extern "C" sepllm_status sepllm_build_index(const sepllm_index_desc* desc,
   if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
   return launch_index(desc, h, token_ids, sep_ids, static_cast<uint8_t*>(index),
                       static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" sepllm_status sepllm_build_index_varlen(const sepllm_index_desc* desc,
+                                                   const int32_t* token_ids,
+                                                   const int32_t* seq_len, const int32_t* sep_ids,
+                                                   void* index, void* scratch, void* stream_) {
+  sepllm_index_header h;
+  sepllm_status st = fill_index_header(desc, &h);
+  if (st != SEPLLM_OK) return st;
+  if (!token_ids || !seq_len || !index || !scratch || (desc->n_sep > 0 && !sep_ids))
+    return SEPLLM_INVALID_ARG;
+  if (!aligned(index, kAlign) || !aligned(scratch, kAlign) || !aligned(token_ids, 4) ||
+      !aligned(seq_len, 4))
+    return SEPLLM_INVALID_ARG;
+  if (desc->B > 65535) return SEPLLM_UNSUPPORTED;
+  return launch_index(desc, h, token_ids, sep_ids, static_cast<uint8_t*>(index),
+                      static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream_), 0, seq_len);
 }
 
 extern "C" sepllm_status sepllm_build_index_fixed_interval(const sepllm_index_desc* desc,

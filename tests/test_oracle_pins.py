@@ -382,6 +382,39 @@ def test_index_invariants(L, a, n, BM, BN):
             assert tl * BN <= wl < (tl + 1) * BN and (th - 1) * BN < wh <= th * BN and z == 0
 
 
+def test_index_with_lengths_is_the_index_of_the_truncated_sequences():
+    """A batch padded to a common length, with its lengths given, must index every sequence as if
+    it stood alone at its own length (valid positions, valid tiles), leave tiles of padding empty,
+    and count nothing behind the end; the prefix-sum version agrees with the loops."""
+    rng = np.random.default_rng(21)
+    B, L, a, n, BM, BN = 5, 300, 3, 17, 32, 16
+    ids = rng.integers(0, 12, size=(B, L)).astype(np.int32)
+    sep = [2, 7]
+    lens = np.array([300, 299, 97, 1, 0], dtype=np.int32)
+    full = orc.build_index(ids, sep, a, n, BM, BN, L, seq_len=lens)
+    fast = orc.build_index_fast(ids, sep, a, n, BM, BN, L, seq_len=lens)
+    for k in ("cnt", "lim", "side_pos", "n_side", "tile_meta", "seq_len"):
+        assert np.array_equal(full[k], fast[k]), k
+    for b in range(B):
+        Lv = int(lens[b])
+        if Lv == 0:
+            assert full["n_side"][b] == 0 and not full["tile_meta"][b].any() and not full["cnt"][b].any()
+            continue
+        alone = orc.build_index(ids[b:b + 1, :Lv], sep, a, n, BM, BN, L)
+        Tv = (Lv + BM - 1) // BM
+        assert np.array_equal(full["cnt"][b, :Lv + 1], alone["cnt"][0])
+        assert (full["cnt"][b, Lv:] == alone["n_side"][0]).all()          # nothing is counted behind the end
+        assert np.array_equal(full["lim"][b, :Lv], alone["lim"][0])
+        assert np.array_equal(full["side_pos"][b], alone["side_pos"][0]) and full["n_side"][b] == alone["n_side"][0]
+        assert np.array_equal(full["tile_meta"][b, :Tv], alone["tile_meta"][0])
+        assert not full["tile_meta"][b, Tv:].any()
+    # without lengths nothing changes
+    plain = orc.build_index(ids, sep, a, n, BM, BN, L)
+    same = orc.build_index(ids, sep, a, n, BM, BN, L, seq_len=np.full(B, L))
+    for k in ("cnt", "lim", "side_pos", "n_side", "tile_meta"):
+        assert np.array_equal(plain[k], same[k])
+
+
 def test_selected_key_gradients_equal_the_all_rows_backward():
     """attn_keys_bwd (used at sizes where not every row can be evaluated) against attn_bwd_head,
     which is pinned above by autograd and finite differences."""

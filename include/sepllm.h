@@ -34,8 +34,11 @@
  *    rows of O, LSE and dQ are not written; their rows of dK and dV are
  *    written as 0), and padded positions are never initial tokens or
  *    separators.
- *  - Supported: d in {64, 128}; Hq a multiple of Hkv; n_neighbor >= 1;
- *    n_init >= 0; index tiles BM = BN = 128 for the attention calls.
+ *  - Supported: d in {64, 80, 96, 112, 128} for the attention calls (rows of
+ *    exactly d elements, no padding in memory; sizes above 64 run in the
+ *    128-wide kernels and cost what d = 128 costs), d in {64, 128} for the
+ *    cache calls; Hq a multiple of Hkv; n_neighbor >= 1; n_init >= 0; index
+ *    tiles BM = BN = 128 for the attention calls.
  */
 #ifndef SEPLLM_H_
 #define SEPLLM_H_

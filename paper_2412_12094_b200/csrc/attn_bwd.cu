@@ -27,14 +27,14 @@ constexpr float kLog2e = 1.4426950408889634f;
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_delta(const __nv_bfloat16* __restrict__ dO, const __nv_bfloat16* __restrict__ O,
-          const float* __restrict__ LSE, float2* __restrict__ stats, size_t rows) {
+          const float* __restrict__ LSE, float2* __restrict__ stats, size_t rows, int d) {
   constexpr int LPR = D / 8;
   const size_t r = (size_t(blockIdx.x) * 256 + threadIdx.x) / LPR;
   const int l = threadIdx.x % LPR;
   float s = 0.f;
-  if (r < rows) {
-    const uint4 a = *reinterpret_cast<const uint4*>(dO + r * D + l * 8);
-    const uint4 b = *reinterpret_cast<const uint4*>(O + r * D + l * 8);
+  if (r < rows && l * 8 < d) {   // rows of d <= D elements
+    const uint4 a = *reinterpret_cast<const uint4*>(dO + r * d + l * 8);
+    const uint4 b = *reinterpret_cast<const uint4*>(O + r * d + l * 8);
     const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
     const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
 #pragma unroll
@@ -64,21 +64,25 @@ struct BwdParams {
   void* dV;
   int32_t* status;
   int B, L, T, Hq, Hkv, n_neighbor, side_cap, cap_pad, grad_fp32, split, pair_heads;
+  int d;                     // row length of Q, K, V, dO and the gradients in memory (<= D)
   float scale, scale_log2;
 };
 
+// n_cols (a multiple of 8): how many of the 32 values lie inside the row.
 __device__ __forceinline__ void store_row_chunk32(void* base, size_t elem_off, int fp32,
-                                                  const float (&v)[32]) {
+                                                  const float (&v)[32], int n_cols = 32) {
   if (fp32) {
     float4* dst = reinterpret_cast<float4*>(static_cast<float*>(base) + elem_off);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    for (int q = 0; q < 8; ++q)
+      if (4 * q < n_cols) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
   } else {
     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + elem_off);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-      dst[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
-                          pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+      if (8 * q < n_cols)
+        dst[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                            pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
   }
 }
 
@@ -299,14 +303,14 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       const int row = it.t * kBM + r;
       const bool row_ok = row < p.L;
       const uint4* src = reinterpret_cast<const uint4*>((u ? dOg : Qg) +
-                                                        (size_t(it.q_plane) * p.L + row) * D);
+                                                        (size_t(it.q_plane) * p.L + row) * p.d);
       const uint32_t dst = tmem + lane_base + (u ? C::kdOt : C::kQt);
 #pragma unroll
       for (int c = 0; c < D / 64; ++c) {
         uint32_t w[32];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          const uint4 v = row_ok ? src[c * 8 + q] : make_uint4(0, 0, 0, 0);
+          const uint4 v = (row_ok && (c * 8 + q) * 8 < p.d) ? src[c * 8 + q] : make_uint4(0, 0, 0, 0);
           w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
         }
         tmem_st32(dst + c * 32, w);
@@ -424,8 +428,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
           float v[32];
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(rr[e]) * p.scale;
-          store_row_chunk32(p.dQ, (size_t(it.q_plane) * p.L + row) * D + u * (D / 2) + c * 32,
-                            p.grad_fp32, v);
+          const int col = u * (D / 2) + c * 32;
+          store_row_chunk32(p.dQ, (size_t(it.q_plane) * p.L + row) * p.d + col, p.grad_fp32, v,
+                            p.d - col);
         }
       }
       w = w_next;
@@ -844,7 +849,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
               }
             }
           }
-          store_row_chunk32(out, (size_t(kv_plane) * p.L + key) * D + c * 32, p.grad_fp32, v);
+          store_row_chunk32(out, (size_t(kv_plane) * p.L + key) * p.d + c * 32, p.grad_fp32, v,
+                            p.d - c * 32);
         }
       }
     }
@@ -876,18 +882,18 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
     constexpr int RPB = 256 / (D / 8);
     bwd_delta<D><<<unsigned((rows + RPB - 1) / RPB), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(dO), static_cast<const __nv_bfloat16*>(O), LSE, stats,
-        rows);
+        rows, d->d);
   }
   record_event(d, 2, stream);
 
   CUtensorMap mq, mdo, mk, mv, mks, mvs;
   sepllm_status st;
   const int64_t L = d->L, nq = int64_t(d->B) * d->Hq, nkv = int64_t(d->B) * d->Hkv;
-  const int64_t cp = lay.cap_pad;
-  if ((st = make_tile_map(&mq, Q, D, L, nq, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mdo, dO, D, L, nq, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mk, K, D, L, nkv, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mv, V, D, L, nkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  const int64_t cp = lay.cap_pad, dr = d->d;  // rows of dr elements; the boxes read zeros from dr to D
+  if ((st = make_tile_map(&mq, Q, dr, L, nq, dr, L * dr, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mdo, dO, dr, L, nq, dr, L * dr, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mk, K, dr, L, nkv, dr, L * dr, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mv, V, dr, L, nkv, dr, L * dr, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mks, Ks, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mvs, Vs, D, cp, nkv, D, cp * D, 128)) != SEPLLM_OK) return st;
 
@@ -907,6 +913,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.status = reinterpret_cast<int32_t*>(ws);
   p.B = d->B;
   p.L = d->L;
+  p.d = d->d;
   p.T = ih.n_tiles;
   p.Hq = d->Hq;
   p.Hkv = d->Hkv;
@@ -917,7 +924,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.split = lay.split;
   const int G = d->Hq / d->Hkv;
   p.pair_heads = (G % 2 == 0) ? 1 : 0;
-  p.scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
+  p.scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(d->d));
   p.scale_log2 = p.scale * kLog2e;
 
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -971,7 +978,7 @@ extern "C" sepllm_status sepllm_attn_bwd(const sepllm_attn_desc* desc,
   // condition the forward recorded stays readable until the caller looks at it.
   if (!(desc->flags & SEPLLM_ATTN_SIDE_READY)) SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
   const uint8_t* idx = static_cast<const uint8_t*>(index);
-  if (desc->d == 64)
+  if (kernel_head_dim(desc->d) == 64)
     return launch_bwd<64>(desc, idesc, ih, dO, Q, K, V, O, LSE, idx, dQ, dK, dV, ws, stream);
   return launch_bwd<128>(desc, idesc, ih, dO, Q, K, V, O, LSE, idx, dQ, dK, dV, ws, stream);
 }

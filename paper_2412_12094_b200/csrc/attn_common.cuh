@@ -44,15 +44,22 @@ struct FwdParams {
   float* LSE;
   int32_t* status;
   int L, T, Hq, Hkv, n_neighbor, side_cap, side_tiles_cap, pair_heads;
+  int d;                     // row length of Q, K, V and O in memory (<= the kernel's D)
   float scale_log2;
 };
+
+// Head sizes between the kernel widths run in the next wider kernel: the tensor maps of Q, K, V and
+// dO describe rows of d elements, so the columns from d up to the kernel's D arrive as zeros (they
+// add nothing to Q K^T, and give zero columns of O, dQ, dK, dV that are never stored); the side
+// buffers and the side-gradient partials have rows of D elements.
+inline int kernel_head_dim(int d) { return d <= 64 ? 64 : 128; }
 
 struct AttnLayout {
   int cap_pad;  // side_cap rounded up to 128 rows
   // forward workspace: status | Kside | Vside
   size_t off_ks, off_vs, fwd_bytes;
   // backward workspace: status | Kside | Vside | row statistics (LSE in log2 units, Delta) |
-  // dKside | dVside, the last two fp32 [split][B][Hkv][cap_pad][d]
+  // dKside | dVside, the last two fp32 [split][B][Hkv][cap_pad][D], D = kernel_head_dim(d)
   size_t off_delta, off_dks, off_dvs, bwd_bytes;
   int split;
 };
@@ -65,8 +72,8 @@ template <int D>
 __global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
                                const __nv_bfloat16* __restrict__ V,
                                const int32_t* __restrict__ side_pos,
-                               const int32_t* __restrict__ n_side, int L, int Hkv, int side_cap,
-                               int cap_pad, __nv_bfloat16* __restrict__ Ks,
+                               const int32_t* __restrict__ n_side, int L, int d, int Hkv,
+                               int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
                                __nv_bfloat16* __restrict__ Vs);
 
 // Forward for groups of four query heads at head size 128: two CTAs of a cluster work on the four
@@ -90,7 +97,7 @@ inline void record_event(const sepllm_attn_desc* d, int i, cudaStream_t stream) 
     cudaEventRecord(static_cast<cudaEvent_t>(d->events[i]), stream);
 }
 
-// Launches the gather of K/V rows at the side positions into Ks / Vs ([B][Hkv][cap_pad][d]).
+// Launches the gather of K/V rows at the side positions into Ks / Vs ([B][Hkv][cap_pad][D]).
 void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
                    const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
                    void* Ks, void* Vs, cudaStream_t stream);

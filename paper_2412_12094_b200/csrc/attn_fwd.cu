@@ -51,12 +51,13 @@ sepllm_status make_tile_map(CUtensorMap* map, const void* base, int d, int64_t r
 // ---------------------------------------------------------------------------
 // grid (ceil(cap_pad / rows_per_block), Hkv, B).  Row r of the side buffer is K/V row
 // side_pos[r]; rows from n_side up to the next multiple of 128 are zero so that the tile holding
-// the last entries contains only finite numbers.
+// the last entries contains only finite numbers.  Source rows have d elements, side rows D >= d
+// (columns from d on are zero).
 template <int D>
 __global__ void __launch_bounds__(256)
 gather_side_kv(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                const int32_t* __restrict__ side_pos, const int32_t* __restrict__ n_side, int L,
-               int Hkv, int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
+               int d, int Hkv, int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
                __nv_bfloat16* __restrict__ Vs) {
   constexpr int LPR = D / 8;
   constexpr int RPB = 256 / LPR;
@@ -69,9 +70,9 @@ gather_side_kv(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restr
   uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
   if (r < ns) {
     const int pos = side_pos[size_t(b) * side_cap + r];
-    if (pos >= 0 && pos < L) {
-      kv = *reinterpret_cast<const uint4*>(K + (plane * L + pos) * D + l * 8);
-      vv = *reinterpret_cast<const uint4*>(V + (plane * L + pos) * D + l * 8);
+    if (pos >= 0 && pos < L && l * 8 < d) {
+      kv = *reinterpret_cast<const uint4*>(K + (plane * L + pos) * d + l * 8);
+      vv = *reinterpret_cast<const uint4*>(V + (plane * L + pos) * d + l * 8);
     }
   }
   *reinterpret_cast<uint4*>(Ks + (plane * cap_pad + r) * D + l * 8) = kv;
@@ -415,7 +416,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       tc_fence_after();
       const float inv_l = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
       if (row < p.L) p.LSE[size_t(q_plane) * p.L + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-      __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * D;
+      __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * p.d;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t oreg[32];
@@ -429,7 +430,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             val.y = pack_bf16(__uint_as_float(oreg[q4 * 8 + 2]) * inv_l, __uint_as_float(oreg[q4 * 8 + 3]) * inv_l);
             val.z = pack_bf16(__uint_as_float(oreg[q4 * 8 + 4]) * inv_l, __uint_as_float(oreg[q4 * 8 + 5]) * inv_l);
             val.w = pack_bf16(__uint_as_float(oreg[q4 * 8 + 6]) * inv_l, __uint_as_float(oreg[q4 * 8 + 7]) * inv_l);
-            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
+            if (c * 32 + q4 * 8 < p.d) *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
           }
         }
       }
@@ -449,7 +450,7 @@ sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id)
     return SEPLLM_INVALID_ARG;
   if (id->B != d->B || id->L != d->L || id->n_neighbor < 1 || id->n_init < 0 || id->side_cap <= 0)
     return SEPLLM_INVALID_ARG;
-  if (d->d != 64 && d->d != 128) return SEPLLM_UNSUPPORTED;
+  if (d->d < 64 || d->d > 128 || d->d % 16 != 0) return SEPLLM_UNSUPPORTED;
   if (id->BM != kBM || id->BN != kBN) return SEPLLM_UNSUPPORTED;
   if (d->grad_dtype != 0 && d->grad_dtype != 1) return SEPLLM_INVALID_ARG;
   if (d->Hq > 65535 || d->B > 65535 || (d->L + kBM - 1) / kBM > 65535) return SEPLLM_UNSUPPORTED;
@@ -459,7 +460,8 @@ sepllm_status check_attn(const sepllm_attn_desc* d, const sepllm_index_desc* id)
 AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
   AttnLayout a;
   a.cap_pad = (id->side_cap + 127) / 128 * 128;
-  const size_t side_bytes = align_up(size_t(d->B) * d->Hkv * a.cap_pad * d->d * 2);
+  const int D = kernel_head_dim(d->d);
+  const size_t side_bytes = align_up(size_t(d->B) * d->Hkv * a.cap_pad * D * 2);
   a.off_ks = kAlign;
   a.off_vs = a.off_ks + side_bytes;
   a.fwd_bytes = a.off_vs + side_bytes;
@@ -467,7 +469,7 @@ AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
   a.off_dks = a.off_delta + align_up(size_t(d->B) * d->Hq * d->L * 2 * sizeof(float));
   a.split = d->Hq / d->Hkv;  // one side-gradient partial per query head of a group
   const size_t side_grad =
-      align_up(size_t(a.split) * d->B * d->Hkv * a.cap_pad * d->d * sizeof(float));
+      align_up(size_t(a.split) * d->B * d->Hkv * a.cap_pad * D * sizeof(float));
   a.off_dvs = a.off_dks + side_grad;
   a.bwd_bytes = a.off_dvs + side_grad;
   return a;
@@ -476,17 +478,17 @@ AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
 void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
                    const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
                    void* Ks, void* Vs, cudaStream_t stream) {
-  if (d->d == 64) {
+  if (kernel_head_dim(d->d) == 64) {
     constexpr int RPB = 256 / (64 / 8);
     gather_side_kv<64><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
-        n_side, d->L, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
+        n_side, d->L, d->d, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
         static_cast<__nv_bfloat16*>(Vs));
   } else {
     constexpr int RPB = 256 / (128 / 8);
     gather_side_kv<128><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
-        n_side, d->L, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
+        n_side, d->L, d->d, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
         static_cast<__nv_bfloat16*>(Vs));
   }
 }
@@ -508,10 +510,10 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
 
   CUtensorMap mq, mk, mv, mks, mvs;
   sepllm_status st;
-  const int64_t L = d->L;
-  if ((st = make_tile_map(&mq, Q, D, L, int64_t(d->B) * d->Hq, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mk, K, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
-  if ((st = make_tile_map(&mv, V, D, L, int64_t(d->B) * d->Hkv, D, L * D, 128)) != SEPLLM_OK) return st;
+  const int64_t L = d->L, dr = d->d;  // rows of dr elements; the boxes read zeros from dr to D
+  if ((st = make_tile_map(&mq, Q, dr, L, int64_t(d->B) * d->Hq, dr, L * dr, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mk, K, dr, L, int64_t(d->B) * d->Hkv, dr, L * dr, 128)) != SEPLLM_OK) return st;
+  if ((st = make_tile_map(&mv, V, dr, L, int64_t(d->B) * d->Hkv, dr, L * dr, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mks, Ks, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
                           int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
   if ((st = make_tile_map(&mvs, Vs, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
@@ -525,6 +527,7 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.LSE = LSE;
   p.status = reinterpret_cast<int32_t*>(ws);
   p.L = d->L;
+  p.d = d->d;
   p.T = ih.n_tiles;
   p.Hq = d->Hq;
   p.Hkv = d->Hkv;
@@ -533,12 +536,12 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.side_tiles_cap = lay.cap_pad / 128;
   const int G = d->Hq / d->Hkv;
   p.pair_heads = (G % 2 == 0) ? 1 : 0;
-  const float scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(D));
+  const float scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(d->d));
   p.scale_log2 = scale * 1.4426950408889634f;
   if (D == 128 && G % 4 == 0) {
     // groups of four query heads: the CTA-pair kernel (K tiles loaded in 64-row halves)
     CUtensorMap mk64, mks64;
-    if ((st = make_tile_map(&mk64, K, D, L, int64_t(d->B) * d->Hkv, D, L * D, 64)) != SEPLLM_OK) return st;
+    if ((st = make_tile_map(&mk64, K, dr, L, int64_t(d->B) * d->Hkv, dr, L * dr, 64)) != SEPLLM_OK) return st;
     if ((st = make_tile_map(&mks64, Ks, D, lay.cap_pad, int64_t(d->B) * d->Hkv, D,
                             int64_t(lay.cap_pad) * D, 64)) != SEPLLM_OK) return st;
     st = launch_fwd_pair(d, p, ih.n_tiles, mq, mk64, mv, mks64, mvs, stream);
@@ -575,7 +578,7 @@ extern "C" sepllm_status sepllm_attn_fwd(const sepllm_attn_desc* desc,
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
-  if (desc->d == 64)
+  if (kernel_head_dim(desc->d) == 64)
     return launch_fwd<64>(desc, idesc, ih, Q, K, V, static_cast<const uint8_t*>(index), O, LSE, ws,
                           stream);
   return launch_fwd<128>(desc, idesc, ih, Q, K, V, static_cast<const uint8_t*>(index), O, LSE, ws,

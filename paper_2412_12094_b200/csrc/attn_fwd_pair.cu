@@ -392,7 +392,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     tc_fence_after();
     const float inv_l = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
     if (row < p.L) p.LSE[size_t(q_plane) * p.L + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-    __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * kD;
+    __nv_bfloat16* orow = p.O + (size_t(q_plane) * p.L + row) * p.d;
 #pragma unroll
     for (int c = 0; c < kD / 32; ++c) {
       uint32_t oreg[32];
@@ -406,7 +406,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
           val.y = pack_bf16(__uint_as_float(oreg[q4 * 8 + 2]) * inv_l, __uint_as_float(oreg[q4 * 8 + 3]) * inv_l);
           val.z = pack_bf16(__uint_as_float(oreg[q4 * 8 + 4]) * inv_l, __uint_as_float(oreg[q4 * 8 + 5]) * inv_l);
           val.w = pack_bf16(__uint_as_float(oreg[q4 * 8 + 6]) * inv_l, __uint_as_float(oreg[q4 * 8 + 7]) * inv_l);
-          *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
+          if (c * 32 + q4 * 8 < p.d) *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = val;
         }
       }
     }

@@ -72,7 +72,7 @@ def test_fwd_pythia_shape_sampled_heads():
 def test_fwd_rejects_unsupported():
     idesc = api.IndexDesc(1, 256, 4, 64, 9, 128, 128, 256)
     with pytest.raises(api.SepllmError) as e:
-        api.sepllm_attn_workspace_bytes(api.AttnDesc(1, 2, 2, 96, 256, 0.0, 0), idesc)
+        api.sepllm_attn_workspace_bytes(api.AttnDesc(1, 2, 2, 72, 256, 0.0, 0), idesc)
     assert e.value.code == api.UNSUPPORTED
     with pytest.raises(api.SepllmError) as e:
         api.sepllm_attn_workspace_bytes(api.AttnDesc(1, 3, 2, 64, 256, 0.0, 0), idesc)

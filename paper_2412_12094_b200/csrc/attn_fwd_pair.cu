@@ -79,7 +79,8 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
   uint64_t* bar_ke = bar_kf + kNST;          // [NST] K stage free
   uint64_t* bar_vf = bar_ke + kNST;          // [NST] (even)
   uint64_t* bar_ve = bar_vf + kNST;          // [NST]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12 + 4 * kNST);
+  uint64_t* bar_tok = bars + 12 + 4 * kNST;  // [2]   slot x may run its exponentials
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_tok + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -103,6 +104,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
       mbar_init(bar_sl + i, rank == 0 ? 5 : 4);
       mbar_init(bar_p + i, rank == 0 ? 5 : 4);
       mbar_init(bar_pv + i, 1);
+      mbar_init(bar_tok + i, 4);
     }
     mbar_init(bar_o, 2);   // one commit from each of the two issuing threads
     for (int i = 0; i < kNST; ++i) {
@@ -335,8 +337,11 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         m_ref = mx;
         rescale = true;
       }
-      // P = 2^(S * scale - m_ref), packed as bf16 pairs over sreg[c][0..15]
+      // P = 2^(S * scale - m_ref), packed as bf16 pairs over sreg[c][0..15].  The two slots take
+      // turns at this block: side by side they halve each other's rate at the special-function
+      // unit, in turn one slot's exponentials run under the other slot's loads, maxima and stores.
       float tile_sum;
+      if (x == 1 || j > 0) wait(bar_tok + x, (x == 1) ? (j & 1) : ((j - 1) & 1));
       {
         const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
         const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
@@ -355,6 +360,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         const float2 sm = unpack_f32x2(add_f32x2(add_f32x2(ps2[0], ps2[1]), add_f32x2(ps2[2], ps2[3])));
         tile_sum = sm.x + sm.y;
       }
+      if (x == 0 || j + 1 < n_tiles) mbar_arrive_warp(bar_tok + (x ^ 1));
       l_sum = l_sum * corr + tile_sum;
 
       // P_x of the previous key tile has been consumed: the buffer is free and O_x is at rest

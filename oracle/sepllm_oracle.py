@@ -26,7 +26,11 @@ Parity unpinned (the paper gives no value that separates the alternatives):
     entry r at position r, query at the last position).  rope_rotate itself is
     pinned to the mathematics (complex-multiplication form, shift invariance,
     norm preservation), and
-  * where the intervals of the fixed-interval variant start (taken: position 0).
+  * where the intervals of the fixed-interval variant start (taken: position 0), and
+  * rows that pack several documents (the paper does not treat them; taken:
+    Eq. 2 inside each document, nothing across a boundary).  Given that
+    reading, packed_mask_matrix, the packed attention and build_index_packed
+    are pinned to the per-document functions.
 """
 from __future__ import annotations
 
@@ -81,6 +85,51 @@ def mask_rows(f: np.ndarray, a: int, n: int, rows: np.ndarray, cols: np.ndarray 
     return (j <= i) & ((j < a) | f[j] | ((i - j) < n))
 
 
+def document_bounds(doc_first: np.ndarray, length: int | None = None):
+    """start[j], end[j] of the document position j belongs to, for a row that
+    holds several documents one after the other: a document begins at position
+    0 and at every j with doc_first[j] != 0 and ends where the next one begins
+    (or at ``length``, the number of tokens in the row).  Positions from
+    ``length`` on are padding: start = end = j (no document)."""
+    doc_first = np.asarray(doc_first)
+    L = doc_first.shape[0]
+    Lv = L if length is None else int(length)
+    start = np.zeros(L, dtype=np.int64)
+    end = np.zeros(L, dtype=np.int64)
+    s = 0
+    for j in range(L):
+        if j >= Lv:
+            start[j] = j
+            continue
+        if j == 0 or doc_first[j]:
+            s = j
+        start[j] = s
+    e = Lv
+    for j in range(L - 1, -1, -1):
+        if j >= Lv:
+            end[j] = j
+            continue
+        end[j] = e
+        if j == 0 or doc_first[j]:
+            e = j
+    return start, end
+
+
+def packed_mask_matrix(f: np.ndarray, doc_first: np.ndarray, a: int, n: int) -> np.ndarray:
+    """Mask of a row that packs several documents.  The paper trains on full
+    rows and does not treat packing; the reading taken: Eq. 2 holds inside each
+    document and nothing is seen across a boundary, so the initial tokens are
+    the first ``a`` tokens of the query's own document and the neighbour window
+    stops at the document's first token."""
+    L = f.shape[0]
+    start, _ = document_bounds(doc_first)
+    i = np.arange(L)[:, None]
+    j = np.arange(L)[None, :]
+    same_doc = start[None, :] == start[:, None]
+    initial = (j - start[None, :]) < a
+    return (j <= i) & same_doc & (initial | f[None, :] | ((i - j) < n))
+
+
 def kept_pairs(f: np.ndarray, a: int, n: int) -> int:
     """Number of ones in M, counted row by row from the predicate."""
     L = f.shape[0]
@@ -128,19 +177,28 @@ def attn_fwd_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, M: np.ndarray,
     return O, LSE, A
 
 
+def _batch_mask(flags, a, n, b, doc_first):
+    """Mask of sequence b: Eq. 2, or its packed form when document boundaries are given."""
+    if doc_first is None:
+        return mask_matrix(flags[b], a, n)
+    return packed_mask_matrix(flags[b], np.asarray(doc_first)[b], a, n)
+
+
 def attn_fwd(Q: np.ndarray, K: np.ndarray, V: np.ndarray, flags: np.ndarray,
-             a: int, n: int, scale: float | None = None):
+             a: int, n: int, scale: float | None = None, doc_first=None):
     """Forward for a batch.  Q [B][Hq][L][d], K,V [B][Hkv][L][d], flags [B][L].
 
     Query head h reads KV head h // (Hq // Hkv).  The mask is the same for all
     heads (Section 3.2, after Eq. 2).  Returns O [B][Hq][L][d], LSE [B][Hq][L].
+    doc_first [B][L] (optional): rows that pack several documents, see
+    packed_mask_matrix.
     """
     B, Hq, L, d = Q.shape
     G = Hq // K.shape[1]
     O = np.zeros((B, Hq, L, d))
     LSE = np.zeros((B, Hq, L))
     for b in range(B):
-        M = mask_matrix(flags[b], a, n)
+        M = _batch_mask(flags, a, n, b, doc_first)
         for h in range(Hq):
             O[b, h], LSE[b, h], _ = attn_fwd_rows(Q[b, h], K[b, h // G], V[b, h // G], M, scale)
     return O, LSE
@@ -174,9 +232,9 @@ def attn_bwd_head(Q, K, V, dO, M, scale: float | None = None):
     return dQ, dK, dV
 
 
-def attn_bwd(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None):
+def attn_bwd(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None, doc_first=None):
     """Backward for a batch; dK and dV are summed over the query heads that
-    share a KV head."""
+    share a KV head.  doc_first: as in attn_fwd."""
     B, Hq, L, d = Q.shape
     Hkv = K.shape[1]
     G = Hq // Hkv
@@ -184,7 +242,7 @@ def attn_bwd(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None):
     dK = np.zeros((B, Hkv, L, d))
     dV = np.zeros((B, Hkv, L, d))
     for b in range(B):
-        M = mask_matrix(flags[b], a, n)
+        M = _batch_mask(flags, a, n, b, doc_first)
         for h in range(Hq):
             q, k, v = attn_bwd_head(Q[b, h], K[b, h // G], V[b, h // G], dO[b, h], M, scale)
             dQ[b, h] = q
@@ -305,7 +363,7 @@ def attn_keys_bwd_blocked(Q, K, V, dO, f, a: int, n: int, keys, scale: float | N
     return dK, dV
 
 
-def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None):
+def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None = None, doc_first=None):
     """Size of the terms behind every gradient entry, for error bounds in tests.
 
     Each entry of dV, dK, dQ is a sum of products (A_ij dO_i, dLambda_ij Q_i,
@@ -333,7 +391,7 @@ def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None 
     sK = np.zeros((B, Hkv, L, d))
     sV = np.zeros((B, Hkv, L, d))
     for b in range(B):
-        M = mask_matrix(flags[b], a, n)
+        M = _batch_mask(flags, a, n, b, doc_first)
         for h in range(Hq):
             hk = h // G
             O, _, A = attn_fwd_rows(Q[b, h], K[b, hk], V[b, hk], M, scale)
@@ -451,6 +509,69 @@ def build_index_fast(token_ids: np.ndarray, sep_ids, a: int, n: int, BM: int, BN
                                -(-win_hi // BN), per_row[b, r0:r1 + 1].sum(), 0]
     return dict(cnt=cnt.astype(np.int32), lim=lim.astype(np.int32), side_pos=side_pos,
                 n_side=cnt[:, L].astype(np.int32), tile_meta=tile_meta, seq_len=lens)
+
+
+def build_index_packed(token_ids: np.ndarray, doc_first: np.ndarray, sep_ids, a: int, n: int,
+                       BM: int, BN: int, side_cap: int, seq_len=None):
+    """Index arrays for rows that pack several documents (packed_mask_matrix).
+
+    Side members are the separators and the first ``a`` tokens of every
+    document; cnt, side_pos, n_side are as in build_index.  With start[i] /
+    end[i] the bounds of row i's document (document_bounds):
+      win_start[i] = max(i-n+1, start[i])   first key of the row's window
+      lim[i]       = cnt[win_start[i]]      side members before the window ...
+      side_lo[i]   = cnt[start[i]]          ... from the document's first one on:
+                                            row i keeps side entries [side_lo, lim)
+    doc_start = start, doc_end = end are part of the index (a key j is kept by
+    queries up to end[j] - 1 only).  tile_meta as in build_index with
+      0 side_full = floor(lim[first row] / BN), 1 side_last = ceil(lim[last row] / BN)
+      2 win_lo = win_start[first row], 3 win_hi = last row + 1, 4, 5 their tiles
+      6 pairs = sum over the tile's valid rows of (lim - side_lo) + (i - win_start + 1)
+      7 side_first = floor(side_lo[first row] / BN)   first side tile any row sees
+    """
+    token_ids = np.asarray(token_ids)
+    doc_first = np.asarray(doc_first)
+    B, L = token_ids.shape
+    T = (L + BM - 1) // BM
+    cnt = np.zeros((B, L + 1), dtype=np.int32)
+    lim = np.zeros((B, L), dtype=np.int32)
+    doc_start = np.zeros((B, L), dtype=np.int32)
+    doc_end = np.zeros((B, L), dtype=np.int32)
+    side_pos = np.full((B, side_cap), -1, dtype=np.int32)
+    n_side = np.zeros((B,), dtype=np.int32)
+    tile_meta = np.zeros((B, T, 8), dtype=np.int32)
+    sep = set(int(x) for x in sep_ids)
+    lens = np.full((B,), L, dtype=np.int32) if seq_len is None else np.asarray(seq_len, dtype=np.int32)
+    for b in range(B):
+        Lv = int(lens[b])
+        start, end = document_bounds(doc_first[b], Lv)
+        doc_start[b], doc_end[b] = start, end
+        k = 0
+        for j in range(L):
+            cnt[b, j] = k
+            if j < Lv and (j - start[j] < a or int(token_ids[b, j]) in sep):
+                if k < side_cap:
+                    side_pos[b, k] = j
+                k += 1
+        cnt[b, L] = k
+        n_side[b] = k
+        win_start = [max(i - n + 1, int(start[i])) for i in range(L)]
+        side_lo = [int(cnt[b, int(start[i])]) for i in range(L)]
+        for i in range(L):
+            lim[b, i] = cnt[b, win_start[i]]
+        for t in range(T):
+            r0 = t * BM
+            if r0 >= Lv:
+                continue
+            r1 = min(Lv, (t + 1) * BM) - 1
+            pairs = 0
+            for i in range(r0, r1 + 1):
+                pairs += int(lim[b, i]) - side_lo[i] + (i - win_start[i] + 1)
+            win_lo, win_hi = win_start[r0], r1 + 1
+            tile_meta[b, t] = [int(lim[b, r0]) // BN, -(-int(lim[b, r1]) // BN), win_lo, win_hi,
+                               win_lo // BN, -(-win_hi // BN), pairs, side_lo[r0] // BN]
+    return dict(cnt=cnt, lim=lim, side_pos=side_pos, n_side=n_side, tile_meta=tile_meta, seq_len=lens,
+                doc_start=doc_start, doc_end=doc_end)
 
 
 # ----------------------------------------------------------------------------

@@ -15,6 +15,9 @@ Recipe
   ("geometric"): a segment of length g is g-1 ordinary tokens followed by its
   separator.
 * Q, K, V, dO: N(0,1) in fp32, rounded to nearest-even bf16.
+* document boundaries of packed rows: document lengths geometric with a given
+  mean (the length mix of a packed pre-training row: many short documents, a
+  few long ones), a 1 at the first token of every document but the first.
 """
 from __future__ import annotations
 
@@ -56,6 +59,21 @@ def token_ids(seed: int, B: int, L: int, rho: float, structure: str = "iid") -> 
     which = SEP_IDS[g.integers(0, SEP_IDS.size, size=(B, L))]
     ids = np.where(is_sep, which, ids).astype(np.int32)
     return ids
+
+
+def doc_first(seed: int, B: int, L: int, mean_len: float) -> np.ndarray:
+    """int32 [B][L]: 1 where a new document begins inside a packed row (position 0 begins one
+    without being marked)."""
+    g = _rng(seed, 9)
+    out = np.zeros((B, L), dtype=np.int32)
+    for b in range(B):
+        pos = 0
+        while True:
+            pos += int(g.geometric(1.0 / mean_len))
+            if pos >= L:
+                break
+            out[b, pos] = 1
+    return out
 
 
 def normal_bf16(seed: int, stream: int, shape) -> torch.Tensor:

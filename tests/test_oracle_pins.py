@@ -12,6 +12,7 @@ import pytest
 import torch
 
 from oracle import sepllm_oracle as orc
+from paper_2412_12094_b200 import inputs
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -526,3 +527,95 @@ def test_rope_decode_pins():
     o_same, l_same = orc.decode_attention_rope(q, K, V, base, q_pos=5, k_pos=np.full(R, 5))
     o_plain, l_plain = orc.decode_attention(q, K, V)
     assert np.allclose(o_same, o_plain, rtol=1e-10, atol=1e-12) and abs(l_same - l_plain) < 1e-10
+
+
+# ----------------------------------------------------------------------------
+# Rows that pack several documents
+# ----------------------------------------------------------------------------
+
+def _docs_of(df):
+    """[(start, end)] of the documents of one row, from the boundary marks alone."""
+    cuts = [0] + [int(j) for j in np.nonzero(df)[0] if j > 0] + [len(df)]
+    return [(cuts[k], cuts[k + 1]) for k in range(len(cuts) - 1) if cuts[k + 1] > cuts[k]]
+
+
+def test_packed_mask_is_the_per_document_mask_on_the_diagonal_blocks():
+    """The packed mask restricted to a document equals Eq. 2's mask of that document alone, and
+    everything outside the diagonal blocks is 0."""
+    for seed, (L, a, n, mean) in enumerate([(60, 2, 5, 9.0), (97, 0, 3, 20.0), (40, 4, 64, 6.0), (33, 1, 1, 1.5)]):
+        ids = inputs.token_ids(40 + seed, 1, L, 0.2)[0]
+        f = orc.separator_flags(ids, inputs.SEP_IDS)
+        df = inputs.doc_first(40 + seed, 1, L, mean)[0]
+        M = orc.packed_mask_matrix(f, df, a, n)
+        expect = np.zeros((L, L), dtype=bool)
+        for s, e in _docs_of(df):
+            expect[s:e, s:e] = orc.mask_matrix(f[s:e], a, n)
+        assert np.array_equal(M, expect)
+    # no boundary marks: the plain mask
+    f = orc.separator_flags(inputs.token_ids(3, 1, 50, 0.2)[0], inputs.SEP_IDS)
+    assert np.array_equal(orc.packed_mask_matrix(f, np.zeros(50, dtype=np.int32), 3, 7), orc.mask_matrix(f, 3, 7))
+
+
+def test_packed_attention_is_attention_on_every_document_by_itself():
+    B, Hq, Hkv, L, d, a, n = 2, 4, 2, 90, 8, 2, 6
+    ids = inputs.token_ids(51, B, L, 0.2)
+    f = np.stack([orc.separator_flags(ids[b], inputs.SEP_IDS) for b in range(B)])
+    df = inputs.doc_first(51, B, L, 14.0)
+    Q, K, V, dO = (t.double().numpy() for t in inputs.qkv_do(51, B, Hq, Hkv, L, d))
+    O, LSE = orc.attn_fwd(Q, K, V, f, a, n, doc_first=df)
+    dQ, dK, dV = orc.attn_bwd(Q, K, V, dO, f, a, n, doc_first=df)
+    for b in range(B):
+        for s, e in _docs_of(df[b]):
+            sl = (slice(b, b + 1), slice(None), slice(s, e))
+            o, lse = orc.attn_fwd(Q[sl], K[sl], V[sl], f[b:b + 1, s:e], a, n, scale=1.0 / np.sqrt(d))
+            assert np.allclose(O[sl], o, atol=1e-12) and np.allclose(LSE[sl], lse, atol=1e-12)
+            q, k, v = orc.attn_bwd(Q[sl], K[sl], V[sl], dO[sl], f[b:b + 1, s:e], a, n, scale=1.0 / np.sqrt(d))
+            assert np.allclose(dQ[sl], q, atol=1e-12) and np.allclose(dK[sl], k, atol=1e-12)
+            assert np.allclose(dV[sl], v, atol=1e-12)
+
+
+def test_packed_index_encodes_the_packed_mask_row_by_row():
+    """Row i of the packed mask is exactly: side entries [cnt[doc_start[i]], lim[i]) plus the keys
+    from max(i-n+1, doc_start[i]) to i; a key j is kept by no query at or after doc_end[j]; the tile
+    words follow from the row values; pairs is the mask's row sum over the tile."""
+    BM = BN = 16
+    for seed, (L, a, n, mean, lens) in enumerate([(150, 2, 7, 23.0, None), (130, 0, 20, 40.0, [101, 130]),
+                                                  (64, 3, 1, 5.0, [64, 17]), (100, 1, 200, 30.0, None)]):
+        B = 2
+        ids = inputs.token_ids(60 + seed, B, L, 0.15)
+        df = inputs.doc_first(60 + seed, B, L, mean)
+        idx = orc.build_index_packed(ids, df, inputs.SEP_IDS, a, n, BM, BN, L, seq_len=lens)
+        for b in range(B):
+            Lv = L if lens is None else lens[b]
+            f = orc.separator_flags(ids[b], inputs.SEP_IDS)
+            M = orc.packed_mask_matrix(f[:Lv], df[b, :Lv], a, n)
+            sp, cnt, lim = idx["side_pos"][b], idx["cnt"][b], idx["lim"][b]
+            ds, de = idx["doc_start"][b], idx["doc_end"][b]
+            for i in range(Lv):
+                ws = max(i - n + 1, int(ds[i]))
+                kept = set(int(x) for x in sp[cnt[ds[i]]:lim[i]]) | set(range(ws, i + 1))
+                assert kept == set(np.nonzero(M[i])[0].tolist()), (seed, b, i)
+                assert len(kept) == (lim[i] - cnt[ds[i]]) + (i - ws + 1)      # the two parts do not overlap
+            for j in range(Lv):
+                assert not M[de[j]:, j].any() and (de[j] == Lv or df[b, de[j]])
+                assert ds[j] == 0 or df[b, ds[j]]
+            for t in range((L + BM - 1) // BM):
+                m = idx["tile_meta"][b, t]
+                r0, r1 = t * BM, min(Lv, (t + 1) * BM) - 1
+                if r0 >= Lv:
+                    assert not m.any()
+                    continue
+                assert m[6] == M[r0:r1 + 1].sum()
+                assert m[0] == lim[r0] // BN and m[1] == -(-lim[r1] // BN) and m[7] == cnt[ds[r0]] // BN
+                assert m[2] == max(r0 - n + 1, ds[r0]) and m[3] == r1 + 1
+                assert m[4] == m[2] // BN and m[5] == -(-m[3] // BN)
+
+
+def test_packed_index_without_boundaries_is_the_plain_index():
+    ids = inputs.token_ids(70, 2, 200, 0.1)
+    plain = orc.build_index(ids, inputs.SEP_IDS, 3, 11, 16, 16, 200, seq_len=[200, 77])
+    packed = orc.build_index_packed(ids, np.zeros_like(ids), inputs.SEP_IDS, 3, 11, 16, 16, 200, seq_len=[200, 77])
+    for k in ("cnt", "side_pos", "n_side", "tile_meta", "seq_len"):
+        assert np.array_equal(plain[k], packed[k]), k
+    # lim differs only on rows of padding, where the packed builder takes cnt at the row itself
+    assert np.array_equal(plain["lim"][0], packed["lim"][0]) and np.array_equal(plain["lim"][1, :77], packed["lim"][1, :77])

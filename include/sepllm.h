@@ -133,7 +133,9 @@ typedef struct {
  *       4 win_tile_lo win_lo / BN
  *       5 win_tile_hi ceil(win_hi / BN)
  *       6 pairs       kept (query,key) pairs in the tile
- *       7 0
+ *       7 side_first  first side tile any row sees (0 unless the index holds documents)
+ *   doc_start [B][L], doc_end [B][L]   bounds of the document each position belongs to; written
+ *       by sepllm_build_index_packed only (the header's `packed` word is then 1)
  * The mask these arrays encode is Eq. 2 with M[i][j] = 1 iff j <= i and
  * (j < n_init or token j is a separator or i - j < n_neighbor).
  */
@@ -145,7 +147,9 @@ typedef struct {
   int32_t n_tiles;     /* ceil(L/BM) */
   int64_t off_cnt, off_lim, off_side_pos, off_n_side, off_tile_meta, total_bytes;
   int64_t off_seq_len;
-  int64_t reserved[19];
+  int64_t off_doc_start, off_doc_end;
+  int64_t packed;      /* 1: built by sepllm_build_index_packed, the document arrays are valid */
+  int64_t reserved[16];
 } sepllm_index_header; /* 256 bytes */
 
 /* Sizes of the index blob and of the scratch buffer sepllm_build_index needs. */
@@ -174,6 +178,27 @@ sepllm_status sepllm_build_index(const sepllm_index_desc* desc, const int32_t* t
 sepllm_status sepllm_build_index_varlen(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* seq_len, const int32_t* sep_ids,
                                         void* index, void* scratch, void* stream);
+
+/* Index of rows that pack several documents one after the other.  The paper
+ * trains on full rows and does not treat packing; the reading taken: Eq. 2
+ * holds inside each document and nothing is seen across a boundary, so the
+ * initial tokens are the first n_init tokens of every document and a row's
+ * neighbour window stops at its document's first token.
+ *   doc_first dev int32 [B][L]: non-zero where a document begins (position 0
+ *             begins one whatever it holds)
+ *   seq_len   dev int32 [B] or NULL (every row full), as for _varlen
+ * Row i then keeps the side entries [cnt[doc_start[i]], lim[i]) and the keys
+ * from max(i-n_neighbor+1, doc_start[i]) to i, with lim[i] = cnt of that first
+ * window key; a key j is kept by queries before doc_end[j] only.  The
+ * attention calls read the header's `packed` word on the device and follow
+ * the document bounds; sepllm_cache_from_prompt takes no such index.
+ * scratch is not used (may be NULL).  Integer output, deterministic; a plain
+ * multi-pass build (one block per row scans it in 1024-token steps), not
+ * tuned like sepllm_build_index. */
+sepllm_status sepllm_build_index_packed(const sepllm_index_desc* desc, const int32_t* token_ids,
+                                        const int32_t* doc_first, const int32_t* seq_len,
+                                        const int32_t* sep_ids, void* index, void* scratch,
+                                        void* stream);
 
 /* Same result as sepllm_build_index, for callers that cannot hand over a scratch
  * buffer because they cannot allocate device memory at the point of the call: a

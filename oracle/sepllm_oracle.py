@@ -406,6 +406,26 @@ def attn_bwd_term_scale(Q, K, V, dO, flags, a: int, n: int, scale: float | None 
     return np.sqrt(sQ), np.sqrt(sK), np.sqrt(sV)
 
 
+def attn_fwd_term_scale(Q, K, V, flags, a: int, n: int, scale: float | None = None, doc_first=None):
+    """Size of the terms behind every entry of O, for error bounds in tests: O_ie
+    is the sum over kept keys j of A_ij V_je, and an implementation that rounds
+    A to bf16 before the product perturbs every term by up to 2^-9 of its size.
+    Returns the root of the sum of the squared terms, [B][Hq][L][d].  (A row
+    that keeps one key has a single term, V itself.)"""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    B, Hq, L, d = Q.shape
+    G = Hq // K.shape[1]
+    out = np.zeros((B, Hq, L, d))
+    for b in range(B):
+        M = _batch_mask(flags, a, n, b, doc_first)
+        for h in range(Hq):
+            _, _, A = attn_fwd_rows(Q[b, h], K[b, h // G], V[b, h // G], M, scale)
+            out[b, h] = np.sqrt((A ** 2) @ (V[b, h // G] ** 2))
+    return out
+
+
 # ----------------------------------------------------------------------------
 # Index (the data the kernels consume; integers, compared bit for bit)
 # ----------------------------------------------------------------------------

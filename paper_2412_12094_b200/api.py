@@ -54,7 +54,8 @@ class IndexHeader(C.Structure):
                 ("desc", IndexDesc), ("n_tiles", C.c_int32),
                 ("off_cnt", C.c_int64), ("off_lim", C.c_int64), ("off_side_pos", C.c_int64),
                 ("off_n_side", C.c_int64), ("off_tile_meta", C.c_int64), ("total_bytes", C.c_int64),
-                ("off_seq_len", C.c_int64), ("reserved", C.c_int64 * 19)]
+                ("off_seq_len", C.c_int64), ("off_doc_start", C.c_int64), ("off_doc_end", C.c_int64),
+                ("packed", C.c_int64), ("reserved", C.c_int64 * 16)]
 
 
 class CacheHeader(C.Structure):
@@ -65,7 +66,8 @@ class CacheHeader(C.Structure):
 
 
 EXPORTS = [
-    "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_varlen", "sepllm_build_index_static",
+    "sepllm_index_bytes", "sepllm_build_index", "sepllm_build_index_varlen", "sepllm_build_index_packed",
+    "sepllm_build_index_static",
     "sepllm_build_index_fixed_interval",
     "sepllm_attn_workspace_bytes", "sepllm_attn_fwd",
     "sepllm_attn_bwd", "sepllm_cache_bytes", "sepllm_cache_init", "sepllm_cache_update",
@@ -150,6 +152,16 @@ def sepllm_build_index_varlen(desc: IndexDesc, token_ids: torch.Tensor, seq_len:
                                            _ptr(scratch), _stream()), "sepllm_build_index_varlen")
 
 
+def sepllm_build_index_packed(desc: IndexDesc, token_ids: torch.Tensor, doc_first: torch.Tensor, seq_len,
+                              sep_ids, index: torch.Tensor):
+    """Index of rows that pack several documents (doc_first [B][L] int32, non-zero where a document
+    begins; seq_len [B] int32 or None)."""
+    arr, p, n = _sep_array(sep_ids)
+    assert n == desc.n_sep
+    _check(lib().sepllm_build_index_packed(C.byref(desc), _ptr(token_ids), _ptr(doc_first), _ptr(seq_len), p,
+                                           _ptr(index), _ptr(None), _stream()), "sepllm_build_index_packed")
+
+
 def sepllm_build_index_static(desc: IndexDesc, token_ids: torch.Tensor, sep_ids, index: torch.Tensor):
     """Index build for callers that cannot allocate a scratch buffer: the library's own fixed
     array is used instead (B * (2 * ceil(L/4096) + 1) <= 65536).  Calls that may overlap on the GPU must be
@@ -185,6 +197,8 @@ def read_index(index: torch.Tensor) -> dict:
         n_side=arr(h.off_n_side, d.B),
         tile_meta=arr(h.off_tile_meta, d.B * T * 8).reshape(d.B, T, 8),
         seq_len=arr(h.off_seq_len, d.B),
+        doc_start=arr(h.off_doc_start, d.B * d.L).reshape(d.B, d.L),
+        doc_end=arr(h.off_doc_end, d.B * d.L).reshape(d.B, d.L),
     )
 
 

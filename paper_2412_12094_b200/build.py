@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libsepllm.so")
-SOURCES = ["index.cu", "cache.cu", "attn_fwd.cu", "attn_fwd_pair.cu", "attn_bwd.cu", "api.cu"]
+SOURCES = ["index.cu", "index_packed.cu", "cache.cu", "attn_fwd.cu", "attn_fwd_pair.cu", "attn_bwd.cu", "api.cu"]
 
 
 def _stale() -> bool:

@@ -56,6 +56,9 @@ struct BwdParams {
   const int32_t* n_side;     // [B]
   const int32_t* tile_meta;  // [B][T][8]
   const int32_t* seq_len;    // [B]
+  const sepllm_index_header* index_header;   // on the device (its `packed` word is read there)
+  const int32_t* doc_start;  // [B][L]   (packed index only)
+  const int32_t* doc_end;    // [B][L]
   const float2* stats;       // [B][Hq][L] (LSE * log2 e, Delta)
   float* dKs;                // [split][B][Hkv][cap_pad][D] fp32 side partials
   float* dVs;
@@ -117,24 +120,27 @@ struct DqCfg {
 
 // One unit of work of the dQ kernel: a query tile of one head.
 struct DqItem {
-  int t, kv_plane, q_plane, b, ns, wlo, n_tiles, side_full;
+  int t, kv_plane, q_plane, b, sbase, ns, wlo, n_tiles;   // key tiles: side [sbase, sbase + ns), window from wlo
+  SlotGeom g;
 };
 // Items are numbered tile-major (longest tiles first), heads x batch minor, so that the heads of
 // a GQA group work on the same K/V tiles at the same time.
-__device__ __forceinline__ DqItem dq_item(const BwdParams& p, int w) {
+__device__ __forceinline__ DqItem dq_item(const BwdParams& p, const DocView& dv, int w) {
   const int hb = p.Hq * p.B;
   const int x = w % hb;
   DqItem it;
   it.b = x / p.Hq;
   const int hq = x % p.Hq;
   it.t = p.T - 1 - w / hb;
-  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, it.b, p.T, it.t, hq, p.cap_pad / kBN);
+  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, it.b, p.T, it.t, hq, p.cap_pad / kBN, dv, p.L,
+                               p.n_neighbor);
   it.kv_plane = it.b * p.Hkv + hq / (p.Hq / p.Hkv);
   it.q_plane = it.b * p.Hq + hq;
-  it.ns = g.ns;
+  it.sbase = (g.t >= 0) ? g.s0 : 0;
+  it.ns = max(0, g.ns - it.sbase);
   it.wlo = g.wlo;
-  it.n_tiles = (g.t >= 0) ? g.ns + (g.whi - g.wlo) : 0;   // 0: a tile of padding, skipped by every role
-  it.side_full = g.side_full;
+  it.n_tiles = (g.t >= 0) ? it.ns + (g.whi - g.wlo) : 0;   // 0: a tile of padding, skipped by every role
+  it.g = g;
   return it;
 }
 
@@ -191,6 +197,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  const DocView dv = doc_view(p.index_header, p.cnt, p.doc_start, p.doc_end);
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (!mbar_wait(bar, parity, abort_flag)) {
@@ -205,10 +212,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       // ---------------- TMA producer ----------------
       int tb = 0;  // tiles before this item
       for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
-        const DqItem it = dq_item(p, w);   // (an empty item has no tiles)
+        const DqItem it = dq_item(p, dv, w);   // (an empty item has no tiles)
         for (int j = 0; j < it.n_tiles; ++j) {
           const bool side = j < it.ns;
-          const int y = side ? j * kBN : (it.wlo + (j - it.ns)) * kBN;
+          const int y = side ? (it.sbase + j) * kBN : (it.wlo + (j - it.ns)) * kBN;
           const int gi = tb + j, st = gi % NST;
           if (gi >= NST) wait(bar_e + st, (gi / NST - 1) & 1);
           mbar_expect_tx(bar_f + st, C::kStage);
@@ -253,7 +260,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       uint32_t fpar = 0;     // parity of that stage's "full" barrier
       uint32_t gpar = 0;     // parity of the per-tile barriers (tile counter & 1)
       for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
-        const int n_tiles = dq_item(p, w).n_tiles;
+        const int n_tiles = dq_item(p, dv, w).n_tiles;
         if (n_tiles == 0) continue;
         wait(bar_qdo, ino & 1);
         wait(bar_f + st, fpar);
@@ -322,35 +329,27 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     int tb = 0, ino = 0;
     // the next item of this CTA that has work, from w on
     auto next_item = [&](int w) {
-      while (w < n_items && dq_item(p, w).n_tiles == 0) w += gridDim.x;
+      while (w < n_items && dq_item(p, dv, w).n_tiles == 0) w += gridDim.x;
       return w;
     };
     int w = next_item(blockIdx.x);
-    if (w < n_items) load_qdo(dq_item(p, w));
+    if (w < n_items) load_qdo(dq_item(p, dv, w));
     for (; w < n_items; ++ino) {
-      const DqItem it = dq_item(p, w);
+      const DqItem it = dq_item(p, dv, w);
       const int w_next = next_item(w + gridDim.x);
       const int t = it.t, ns = it.ns;
       const int row = t * kBM + r;
       const bool row_ok = row < p.L;
       // ---------------- dS: warpgroup u takes key columns [64u, 64u+64) of every tile ---------
-      const int lim_i = row_ok ? min(p.lim[size_t(it.b) * p.L + row], p.side_cap) : 0;
+      const RowGeom rg = row_geom(p.lim, dv, it.b, p.L, row, p.n_neighbor, p.side_cap);
       const float2 stt = row_ok ? p.stats[size_t(it.q_plane) * p.L + row] : make_float2(INFINITY, 0.f);
       const float neg_lse2 = -stt.x, delta_i = stt.y;
       for (int j = 0; j < it.n_tiles; ++j) {
         const int gi = tb + j;
         const bool side = j < ns;
-        int c_lo = 0, c_hi = kBN;
+        int c_lo, c_hi;
         bool need_mask;
-        if (side) {
-          c_hi = lim_i - j * kBN;
-          need_mask = (j >= it.side_full);
-        } else {
-          const int key0 = (it.wlo + (j - ns)) * kBN;
-          c_hi = row - key0 + 1;
-          c_lo = row - p.n_neighbor + 1 - key0;
-          need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-        }
+        key_range(side, side ? it.sbase + j : it.wlo + (j - ns), it.g, row, rg, c_lo, c_hi, need_mask);
         // phase A (needs S only; runs under the previous tile's dQ and this tile's dP MMAs):
         // P = exp2(S * scale - LSE), kept in registers
         wait(bar_s, gi & 1);
@@ -410,7 +409,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       tb += it.n_tiles;
       // Every S and dP MMA of this item is complete (the last dP was waited for), so Q and dO of
       // the next item can go into tensor memory while this item's last dQ MMAs run.
-      if (w_next < n_items) load_qdo(dq_item(p, w_next));
+      if (w_next < n_items) load_qdo(dq_item(p, dv, w_next));
       // ---------------- epilogue: each warpgroup stores half of the row ----------------
       wait(bar_acc, ino & 1);
       tc_fence_after();
@@ -520,15 +519,28 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   // query tiles [t_lo, t_hi] that keep at least one key of this tile; tiles of padding behind
   // the sequence's last token (seq_len from the index) are left out
-  const int t_last = (p.seq_len[b] + kBM - 1) / kBM - 1;
-  int t_lo, t_hi;
+  // With document bounds (a packed index) a key is kept by the queries of its own document only:
+  // q_end_first / q_end_last are the ends of the documents of the tile's first and last key.
+  const DocView dv = doc_view(p.index_header, p.cnt, p.doc_start, p.doc_end);
+  const int len = p.seq_len[b];
+  const int t_last = (len + kBM - 1) / kBM - 1;
+  int t_lo, t_hi, q_end_first = kFar;
   if (SIDE) {
     if (kt * kBN >= ns) return;  // no entries in this side tile: nothing reads its partial rows
-    t_lo = (p.side_pos[size_t(b) * p.side_cap + kt * kBN] + p.n_neighbor) / kBM;
+    const int32_t* sp = p.side_pos + size_t(b) * p.side_cap;
+    t_lo = (sp[kt * kBN] + p.n_neighbor) / kBM;
     t_hi = t_last;
+    if (dv.doc_end) {
+      q_end_first = dv.doc_end[size_t(b) * p.L + sp[kt * kBN]];
+      t_hi = min(t_last, (dv.doc_end[size_t(b) * p.L + sp[min(ns, kt * kBN + kBN) - 1]] - 1) / kBM);
+    }
   } else {
     t_lo = kt;  // kBM == kBN
     t_hi = min(t_last, (kt * kBN + kBN - 1 + p.n_neighbor - 1) / kBM);
+    if (dv.doc_end && kt * kBN < len) {
+      q_end_first = dv.doc_end[size_t(b) * p.L + kt * kBN];
+      t_hi = min(t_hi, (dv.doc_end[size_t(b) * p.L + min(len, kt * kBN + kBN) - 1] - 1) / kBM);
+    }
   }
   const int n_it = max(0, t_hi - t_lo + 1) * n_g;
 
@@ -700,26 +712,29 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
     const uint32_t tST = tmem + lane_base + C::kST + u * 64;
     const uint32_t tdPT = tmem + lane_base + C::kdPT + u * 64;
-    // queries that keep this key: [q_first, q_first + span)
-    int q_first, span, tile_q_max;
+    // queries that keep this key: [q_first, q_end)
+    int q_first, q_end, tile_q_max;
     if (SIDE) {
-      q_first = (key < ns) ? p.side_pos[size_t(b) * p.side_cap + key] + p.n_neighbor : kFar;
-      span = kFar;
+      const int pos = (key < ns) ? p.side_pos[size_t(b) * p.side_cap + key] : -1;
+      q_first = (pos >= 0) ? pos + p.n_neighbor : kFar;
+      q_end = (pos >= 0 && dv.doc_end) ? dv.doc_end[size_t(b) * p.L + pos] : kFar;
       // first query that keeps every key of the tile (never, if the tile has padding rows)
       tile_q_max = (kt * kBN + kBN <= ns)
                        ? p.side_pos[size_t(b) * p.side_cap + kt * kBN + kBN - 1] + p.n_neighbor
                        : kFar;
     } else {
       q_first = key;
-      span = p.n_neighbor;
+      q_end = key + p.n_neighbor;
+      if (dv.doc_end && key < p.L) q_end = min(q_end, dv.doc_end[size_t(b) * p.L + key]);
       tile_q_max = 0;
     }
     for (int it = 0; it < n_it; ++it) {
       const int q0 = q0_of(it);
-      const int c_lo = q_first - q0, c_hi = c_lo + span;
+      const int c_lo = q_first - q0, c_hi = q_end - q0;
       bool need_mask;
       if (SIDE) need_mask = tile_q_max > q0;
       else need_mask = !(kt * kBN + kBN - 1 <= q0 && q0 + kBM - 1 <= kt * kBN + p.n_neighbor - 1);
+      need_mask = need_mask || (q0 + kBM > q_end_first);   // a document of the tile ends inside these queries
       // phase A (needs S^T only; runs under the previous iteration's dV / dK and this iteration's
       // dP^T MMAs): P^T = exp2(S^T * scale - LSE), kept in registers
       wait(bar_sf, it & 1);
@@ -904,6 +919,9 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.n_side = n_side;
   p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
   p.seq_len = reinterpret_cast<const int32_t*>(index + ih.off_seq_len);
+  p.index_header = reinterpret_cast<const sepllm_index_header*>(index);
+  p.doc_start = reinterpret_cast<const int32_t*>(index + ih.off_doc_start);
+  p.doc_end = reinterpret_cast<const int32_t*>(index + ih.off_doc_end);
   p.stats = stats;
   p.dKs = reinterpret_cast<float*>(ws + lay.off_dks);
   p.dVs = reinterpret_cast<float*>(ws + lay.off_dvs);

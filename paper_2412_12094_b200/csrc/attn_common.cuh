@@ -7,16 +7,39 @@ namespace sepllm {
 constexpr int kBM = 128, kBN = 128;
 constexpr uint32_t kTileBlockBytes = 128 * 128;  // 128 rows x 64 bf16, one swizzled block
 
+// Document bounds of an index built for rows that pack several documents
+// (sepllm_build_index_packed); all null for any other index.  With them, row i keeps the side
+// entries [cnt[doc_start[i]], lim[i]) and the keys from max(i - n + 1, doc_start[i]) to i, and key
+// j is kept by queries before doc_end[j] only.
+struct DocView {
+  const int32_t* cnt;        // [B][L+1]
+  const int32_t* doc_start;  // [B][L]
+  const int32_t* doc_end;    // [B][L]
+};
+__device__ __forceinline__ DocView doc_view(const sepllm_index_header* hdr, const int32_t* cnt,
+                                            const int32_t* doc_start, const int32_t* doc_end) {
+  DocView v;
+  const bool packed = hdr->packed != 0;
+  v.cnt = packed ? cnt : nullptr;
+  v.doc_start = packed ? doc_start : nullptr;
+  v.doc_end = packed ? doc_end : nullptr;
+  return v;
+}
+
 // One query tile of a two-slot CTA (forward and dQ kernels): tile index (-1 = empty slot), query
-// head, and the tile's key ranges from tile_meta.
+// head, and the tile's key ranges from tile_meta: side tiles [s0, ns) of which those in
+// [full_lo, side_full) are kept in full by every row, window tiles [wlo, whi); ws_last is the
+// first window key of the tile's last row.
 struct SlotGeom {
-  int t, hq, side_full, ns, wlo, whi;
+  int t, hq, side_full, ns, wlo, whi, s0, full_lo, ws_last;
 };
 // A tile that starts at or behind the end of its sequence (seq_len from the index) is empty too.
 __device__ __forceinline__ SlotGeom load_slot(const int32_t* tile_meta, const int32_t* seq_len, int b,
-                                              int T, int t, int hq, int side_tiles_cap) {
+                                              int T, int t, int hq, int side_tiles_cap,
+                                              const DocView& dv, int L, int n_neighbor) {
   SlotGeom g;
-  g.t = (t >= 0 && t * kBM < seq_len[b]) ? t : -1;
+  const int len = seq_len[b];
+  g.t = (t >= 0 && t * kBM < len) ? t : -1;
   g.hq = hq;
   if (g.t >= 0) {
     const int32_t* meta = tile_meta + (size_t(b) * T + t) * 8;
@@ -24,22 +47,74 @@ __device__ __forceinline__ SlotGeom load_slot(const int32_t* tile_meta, const in
     g.ns = min(meta[1], side_tiles_cap);
     g.wlo = meta[4];
     g.whi = meta[5];
+    g.s0 = 0;
+    g.full_lo = 0;
+    g.ws_last = t * kBM + kBM - n_neighbor;
+    if (dv.doc_start) {
+      const int r1 = min(len, (t + 1) * kBM) - 1;
+      const int s = dv.doc_start[size_t(b) * L + r1];
+      g.s0 = min(meta[7], g.ns);
+      g.full_lo = (dv.cnt[size_t(b) * (L + 1) + s] + kBN - 1) / kBN;
+      g.ws_last = max(r1 - n_neighbor + 1, s);
+    }
   } else {
     g.side_full = 0; g.ns = 0; g.wlo = 0x3fffffff; g.whi = 0;
+    g.s0 = 0x3fffffff; g.full_lo = 0; g.ws_last = 0;
   }
   return g;
 }
-// Key tile j of the CTA's list (side tiles [0, ns), then window tiles from wlo) is kept by slot g.
-__device__ __forceinline__ bool slot_active(const SlotGeom& g, int ns, int wlo, int j) {
-  if (j < ns) return j < g.ns;
-  const int w = wlo + (j - ns);
+// Key tile j of the CTA's list (side tiles sbase .. sbase + nsl - 1, then window tiles from wlo)
+// is kept by slot g.
+__device__ __forceinline__ bool slot_active(const SlotGeom& g, int sbase, int nsl, int wlo, int j) {
+  if (j < nsl) return sbase + j >= g.s0 && sbase + j < g.ns;
+  const int w = wlo + (j - nsl);
   return w >= g.wlo && w < g.whi;
 }
 
+// What one query row keeps: side entries [lo, lim), window keys [ws, row].
+struct RowGeom {
+  int lim, lo, ws;
+};
+__device__ __forceinline__ RowGeom row_geom(const int32_t* lim, const DocView& dv, int b, int L,
+                                            int row, int n_neighbor, int side_cap) {
+  RowGeom r;
+  r.lim = 0;
+  r.lo = 0;
+  r.ws = row - n_neighbor + 1;
+  if (row < L) {
+    r.lim = min(lim[size_t(b) * L + row], side_cap);
+    if (dv.doc_start) {
+      const int s = dv.doc_start[size_t(b) * L + row];
+      r.lo = min(dv.cnt[size_t(b) * (L + 1) + s], side_cap);
+      r.ws = max(r.ws, s);
+    }
+  }
+  return r;
+}
+// Kept columns [c_lo, c_hi) of one key tile for one row, and whether any row of the query tile
+// needs the mask at all.  tile: side tile index, or window tile index (keys tile*kBN ...).
+__device__ __forceinline__ void key_range(bool side, int tile, const SlotGeom& g, int row,
+                                          const RowGeom& rg, int& c_lo, int& c_hi, bool& need_mask) {
+  const int k0 = tile * kBN;
+  if (side) {
+    c_lo = rg.lo - k0;
+    c_hi = rg.lim - k0;
+    need_mask = (tile >= g.side_full) || (tile < g.full_lo);
+  } else {
+    c_lo = rg.ws - k0;
+    c_hi = row - k0 + 1;
+    need_mask = (k0 + kBN - 1 > g.t * kBM) || (k0 < g.ws_last);
+  }
+}
+
 struct FwdParams {
+  const sepllm_index_header* index_header;   // on the device (its `packed` word is read there)
+  const int32_t* cnt;        // [B][L+1]
   const int32_t* lim;        // [B][L]
   const int32_t* tile_meta;  // [B][T][8]
   const int32_t* seq_len;    // [B]
+  const int32_t* doc_start;  // [B][L]   (packed index only)
+  const int32_t* doc_end;    // [B][L]
   __nv_bfloat16* O;
   float* LSE;
   int32_t* status;

@@ -144,19 +144,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 
   // the two slots of this CTA (a slot is empty when its tile does not exist or holds only padding)
   SlotGeom g0, g1;
+  const DocView dv = doc_view(p.index_header, p.cnt, p.doc_start, p.doc_end);
   if (p.pair_heads) {
     const int t = p.T - 1 - int(blockIdx.y);
-    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx + 1, p.side_tiles_cap);
+    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap, dv, p.L, p.n_neighbor);
+    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx + 1, p.side_tiles_cap, dv, p.L, p.n_neighbor);
   } else {
     const int t = p.T - 1 - 2 * int(blockIdx.y);
-    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t - 1, hx, p.side_tiles_cap);
-    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, hx, p.side_tiles_cap);
+    g0 = load_slot(p.tile_meta, p.seq_len, b, p.T, t - 1, hx, p.side_tiles_cap, dv, p.L, p.n_neighbor);
+    g1 = load_slot(p.tile_meta, p.seq_len, b, p.T, t, hx, p.side_tiles_cap, dv, p.L, p.n_neighbor);
   }
   if (g0.t < 0 && g1.t < 0) return;   // both tiles are padding: nothing to do, nothing written
   const int kv_plane = b * p.Hkv + g1.hq / G;
-  // key tiles of the CTA: side tiles [0, ns), then window tiles [wlo, whi)
-  const int ns = max(g0.ns, g1.ns);
+  // key tiles of the CTA: side tiles [sbase, sbase + ns), then window tiles [wlo, whi)
+  const int sbase = min(g0.s0, g1.s0);
+  const int ns = max(0, max(g0.ns, g1.ns) - sbase);
   const int wlo = min(g0.wlo, g1.wlo);
   const int whi = max(g0.whi, g1.whi);
   const int n_tiles = ns + (whi - wlo);
@@ -211,7 +213,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       for (int j = 0; j < n_tiles; ++j) {
         const int st = j % NST, use = j / NST;
         const bool side = j < ns;
-        const int y = side ? j * kBN : (wlo + (j - ns)) * kBN;
+        const int y = side ? (sbase + j) * kBN : (wlo + (j - ns)) * kBN;
         if (use > 0) wait(bar_ke + st, (use - 1) & 1);
         mbar_expect_tx(bar_kf + st, C::kTile);
         for (int nb = 0; nb < NB; ++nb)
@@ -242,7 +244,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         for (int x = 0; x < 2; ++x) {
           const SlotGeom& g = x ? g1 : g0;
           const uint32_t tS = tmem + (x ? C::kS1 : C::kS0), tO = tmem + (x ? C::kO1 : C::kO0);
-          if (s >= 1 && slot_active(g, ns, wlo, s - 1)) {
+          if (s >= 1 && slot_active(g, sbase, ns, wlo, s - 1)) {
             const int j = s - 1, st = j % NST;
             wait(bar_p + x, n_pv[x] & 1);
             if (!v_waited) { wait(bar_vf + st, (j / NST) & 1); v_waited = true; }
@@ -254,7 +256,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
               umma_ts_lo(tO, tS + k * 8, v_lo + mnmajor_step(k), idesc_o, 1);
             ++n_pv[x];
           }
-          if (s < n_tiles && slot_active(g, ns, wlo, s)) {
+          if (s < n_tiles && slot_active(g, sbase, ns, wlo, s)) {
             const int st = s % NST;
             if (!q_seen[x]) { wait(bar_q + x, 0); q_seen[x] = true; }
             if (!k_waited) { wait(bar_kf + st, (s / NST) & 1); k_waited = true; }
@@ -286,14 +288,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (t >= 0) {
       const int row = t * kBM + r;  // this thread's query position
       const int q_plane = b * p.Hq + g.hq;
-      const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-      const int side_full = g.side_full;
+      const RowGeom rg = row_geom(p.lim, dv, b, p.L, row, p.n_neighbor, p.side_cap);
       float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
       float l_sum = 0.f;
       int n_done = 0;
       uint32_t sreg[4][32];
       for (int j = 0; j < n_tiles; ++j) {
-        if (!slot_active(g, ns, wlo, j)) continue;
+        if (!slot_active(g, sbase, ns, wlo, j)) continue;
         wait(bar_s + x, n_done & 1);
         tc_fence_after();
         // MMAs complete in issue order: S of slot 1 for tile j done means both slots' S MMAs have
@@ -308,17 +309,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 
         // kept columns of this tile for this row: [c_lo, c_hi)
         const bool side = j < ns;
-        int c_lo = 0, c_hi = kBN;
+        int c_lo, c_hi;
         bool need_mask;
-        if (side) {
-          c_hi = lim_i - j * kBN;
-          need_mask = (j >= side_full);
-        } else {
-          const int key0 = (wlo + (j - ns)) * kBN;
-          c_hi = row - key0 + 1;
-          c_lo = row - p.n_neighbor + 1 - key0;
-          need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-        }
+        key_range(side, side ? sbase + j : wlo + (j - ns), g, row, rg, c_lo, c_hi, need_mask);
         // Reference exponent.  A tile that needs no mask and finds a reference already set skips
         // the maximum: its exponentials are taken against the old reference, which is exact as
         // long as nothing overflows (fp32 sums and bf16 P have the range for a lag of 2^64), and
@@ -520,9 +513,13 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
                           int64_t(lay.cap_pad) * D, 128)) != SEPLLM_OK) return st;
 
   FwdParams p;
+  p.index_header = reinterpret_cast<const sepllm_index_header*>(index);
+  p.cnt = reinterpret_cast<const int32_t*>(index + ih.off_cnt);
   p.lim = reinterpret_cast<const int32_t*>(index + ih.off_lim);
   p.tile_meta = reinterpret_cast<const int32_t*>(index + ih.off_tile_meta);
   p.seq_len = reinterpret_cast<const int32_t*>(index + ih.off_seq_len);
+  p.doc_start = reinterpret_cast<const int32_t*>(index + ih.off_doc_start);
+  p.doc_end = reinterpret_cast<const int32_t*>(index + ih.off_doc_end);
   p.O = static_cast<__nv_bfloat16*>(O);
   p.LSE = LSE;
   p.status = reinterpret_cast<int32_t*>(ws);

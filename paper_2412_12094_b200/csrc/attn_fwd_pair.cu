@@ -92,9 +92,12 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
   const int t = p.T - 1 - int(blockIdx.y);
   const int G = p.Hq / p.Hkv;
   if (t * kBM >= p.seq_len[b]) return;   // a tile of padding (the same for both CTAs of the pair)
-  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap);
+  const DocView dv = doc_view(p.index_header, p.cnt, p.doc_start, p.doc_end);
+  const SlotGeom g = load_slot(p.tile_meta, p.seq_len, b, p.T, t, 2 * hx, p.side_tiles_cap, dv, p.L,
+                               p.n_neighbor);
   const int kv_plane = b * p.Hkv + (2 * hx) / G;
-  const int ns = g.ns, wlo = g.wlo;
+  // key tiles: side tiles [sbase, sbase + ns), then window tiles [wlo, whi)
+  const int sbase = g.s0, ns = max(0, g.ns - g.s0), wlo = g.wlo;
   const int n_tiles = ns + (g.whi - g.wlo);
 
   if (tid == 0) {
@@ -164,7 +167,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
       for (int j = 0; j < n_tiles; ++j) {
         const int st = j % kNST, use = j / kNST;
         const bool side = j < ns;
-        const int y = side ? j * kBN : (wlo + (j - ns)) * kBN;
+        const int y = side ? (sbase + j) * kBN : (wlo + (j - ns)) * kBN;
         // K: this CTA's 64 keys of the tile, all 128 columns
         if (use > 0) wait(bar_ke + st, (use - 1) & 1);
         if (rank == 0) mbar_expect_tx(bar_kf + st, 2 * kKHalf);
@@ -280,8 +283,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     const int hq = 2 * hx + x;
     const int row = t * kBM + r;  // this thread's query position
     const int q_plane = b * p.Hq + hq;
-    const int lim_i = (row < p.L) ? min(p.lim[size_t(b) * p.L + row], p.side_cap) : 0;
-    const int side_full = g.side_full;
+    const RowGeom rg = row_geom(p.lim, dv, b, p.L, row, p.n_neighbor, p.side_cap);
     float m_ref = -INFINITY;  // reference exponent (log2 units), may lag the true row maximum
     float l_sum = 0.f;
     uint32_t sreg[4][32];
@@ -296,17 +298,9 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 
       // kept columns of this tile for this row: [c_lo, c_hi)
       const bool side = j < ns;
-      int c_lo = 0, c_hi = kBN;
+      int c_lo, c_hi;
       bool need_mask;
-      if (side) {
-        c_hi = lim_i - j * kBN;
-        need_mask = (j >= side_full);
-      } else {
-        const int key0 = (wlo + (j - ns)) * kBN;
-        c_hi = row - key0 + 1;
-        c_lo = row - p.n_neighbor + 1 - key0;
-        need_mask = (key0 + kBN - 1 > t * kBM) || (key0 < t * kBM + kBM - p.n_neighbor);
-      }
+      key_range(side, side ? sbase + j : wlo + (j - ns), g, row, rg, c_lo, c_hi, need_mask);
       if (need_mask) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)

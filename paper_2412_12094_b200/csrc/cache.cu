@@ -322,7 +322,8 @@ prompt_plan(sepllm_cache_header h, uint8_t* __restrict__ state, const uint8_t* _
     const sepllm_index_header* dev = reinterpret_cast<const sepllm_index_header*>(index);
     bool bad = dev->magic != SEPLLM_INDEX_MAGIC || dev->desc.B != ih.desc.B ||
                dev->desc.L != ih.desc.L || dev->desc.n_init != ih.desc.n_init ||
-               dev->desc.side_cap != ih.desc.side_cap;
+               dev->desc.side_cap != ih.desc.side_cap ||
+               dev->packed != 0;   // an index of packed rows describes no single prompt
     int T = L;
     if (prompt_len) {
       T = prompt_len[b];

@@ -407,6 +407,10 @@ sepllm_status fill_index_header(const sepllm_index_desc* d, sepllm_index_header*
   off = align_up(off + sizeof(int32_t) * size_t(d->B) * h->n_tiles * 8);
   h->off_seq_len = off;
   off = align_up(off + sizeof(int32_t) * size_t(d->B));
+  h->off_doc_start = off;
+  off = align_up(off + sizeof(int32_t) * size_t(d->B) * d->L);
+  h->off_doc_end = off;
+  off = align_up(off + sizeof(int32_t) * size_t(d->B) * d->L);
   h->total_bytes = off;
   return SEPLLM_OK;
 }

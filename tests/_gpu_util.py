@@ -96,3 +96,18 @@ def attn_bwd(dO, Q, K, V, O, LSE, idesc, index, grad_dtype=0, scale=0.0):
 
 def flags_of(ids_np, sep_ids):
     return np.isin(ids_np, np.asarray(sep_ids))
+
+
+def assert_o_close(got, ref, rss, what=""):
+    """Entries of O against the oracle: the absolute bound of the parity bar, raised only for
+    entries whose own terms are so large that the bf16 rounding of the weights (rss from
+    oracle.attn_fwd_term_scale) and of the bf16 output exceeds it -- rows that keep one or two
+    keys return (nearly) a V row itself, entries of 3 and 4 among them, and inputs made of many
+    short documents hold hundreds of such rows.  Relative Frobenius error as everywhere else."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    tol = np.maximum(TOL_O["max_abs"], K_ROUND * 2.0 ** -9 * np.asarray(rss) + 2.0 ** -9 * np.abs(ref))
+    worst = float((np.abs(got - ref) / tol).max()) if got.size else 0.0
+    assert worst <= 1.0, f"{what}: an entry is off by {worst:.2f} x its bound"
+    assert errors(got, ref)[1] <= TOL_O["rel_fro"], (what, errors(got, ref))

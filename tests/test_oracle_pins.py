@@ -619,3 +619,20 @@ def test_packed_index_without_boundaries_is_the_plain_index():
         assert np.array_equal(plain[k], packed[k]), k
     # lim differs only on rows of padding, where the packed builder takes cnt at the row itself
     assert np.array_equal(plain["lim"][0], packed["lim"][0]) and np.array_equal(plain["lim"][1, :77], packed["lim"][1, :77])
+
+
+def test_forward_term_scale_is_the_root_sum_square_of_the_terms_of_O():
+    B, Hq, Hkv, L, d, a, n = 1, 2, 1, 40, 6, 2, 5
+    ids = inputs.token_ids(90, B, L, 0.2)
+    f = np.stack([orc.separator_flags(ids[b], inputs.SEP_IDS) for b in range(B)])
+    Q, K, V, _ = (t.double() for t in inputs.qkv_do(90, B, Hq, Hkv, L, d))
+    rss = orc.attn_fwd_term_scale(Q.numpy(), K.numpy(), V.numpy(), f, a, n)
+    M = torch.from_numpy(orc.mask_matrix(f[0], a, n))
+    for h in range(Hq):
+        S = (Q[0, h] @ K[0, 0].T) / math.sqrt(d)
+        A = torch.softmax(S.masked_fill(~M, float("-inf")), dim=-1)
+        terms = A[:, :, None] * V[0, 0][None, :, :]          # [i][j][e]
+        assert np.allclose(rss[0, h], terms.pow(2).sum(1).sqrt().numpy(), rtol=1e-12, atol=1e-15)
+        assert np.allclose(terms.sum(1).numpy(), orc.attn_fwd(Q.numpy(), K.numpy(), V.numpy(), f, a, n)[0][0, h])
+    # a row with one key: the single term is V itself
+    assert np.allclose(rss[0, :, 0], np.abs(V[0, 0, 0].numpy())[None, :])

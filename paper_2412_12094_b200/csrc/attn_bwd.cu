@@ -148,12 +148,14 @@ __device__ __forceinline__ DqItem dq_item(const BwdParams& p, const DocView& dv,
 // barrier phases run on a tile count that continues across items; the next item's Q and dO go
 // into tensor memory as soon as the current item's last S / dP MMAs are complete, and its first
 // MMAs run while the current item's dQ is still being stored.
-template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
-bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
-              const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
-              const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ dOg,
-              const BwdParams p, const int n_items) {
+// PACKED: the index holds document bounds.  The kernel proper picks one of the two bodies by the
+// index header's `packed` word; without the bounds every test for them is compiled out (as
+// run-time tests they cost this kernel, which decodes an item in every role, 8 % of its time).
+template <int D, bool PACKED>
+__device__ __forceinline__ void
+bwd_dq_body(const CUtensorMap& mapK, const CUtensorMap& mapV, const CUtensorMap& mapKs,
+            const CUtensorMap& mapVs, const __nv_bfloat16* __restrict__ Qg,
+            const __nv_bfloat16* __restrict__ dOg, const BwdParams& p, const int n_items) {
   using C = DqCfg<D>;
   constexpr int NB = C::NB, NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
@@ -197,7 +199,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  const DocView dv = doc_view(p.index_header, p.cnt, p.doc_start, p.doc_end);
+  const DocView dv = PACKED ? DocView{p.cnt, p.doc_start, p.doc_end} : DocView{nullptr, nullptr, nullptr};
   bool ok = true;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (!mbar_wait(bar, parity, abort_flag)) {
@@ -438,6 +440,16 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+              const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
+              const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ dOg,
+              const BwdParams p, const int n_items) {
+  if (p.index_header->packed) bwd_dq_body<D, true>(mapK, mapV, mapKs, mapVs, Qg, dOg, p, n_items);
+  else bwd_dq_body<D, false>(mapK, mapV, mapKs, mapVs, Qg, dOg, p, n_items);
 }
 
 // ---------------------------------------------------------------------------

@@ -612,7 +612,7 @@ def main():
     # bwd_dkv_kernel<side> as captured; None for anything else.
     traffic = None
     if dom == "bwd_dkv_kernel<side>" and cfg["d"] == 128 and cfg["Hq"] == 32 and cfg["B"] == 1:
-        traffic = (647.52e6 + 39.84e6) * side_iters / 836.0
+        traffic = (686.49e6 + 39.55e6) * side_iters / 836.0
     out["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                        "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
                        "peak_kind": f"bf16 sustained, {peaks['source']}",

@@ -541,7 +541,7 @@ constexpr int decode_smem_bytes() {
 // then carries the softmax state of rows frow and frow + 8); narrower groups leave the upper
 // half zero and skip its arithmetic.
 template <int D, bool ROPE, bool WIDE>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, 3)   // three CTAs per SM: at most 168 registers
 decode_split(sepllm_cache_header h, float scale_log2, const __nv_bfloat16* __restrict__ q_in,
              const uint8_t* __restrict__ state, const __nv_bfloat16* __restrict__ Kc,
              const __nv_bfloat16* __restrict__ Vc, float* __restrict__ part_ml,

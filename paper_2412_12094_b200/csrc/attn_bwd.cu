@@ -148,8 +148,8 @@ __device__ __forceinline__ DqItem dq_item(const BwdParams& p, const DocView& dv,
 // barrier phases run on a tile count that continues across items; the next item's Q and dO go
 // into tensor memory as soon as the current item's last S / dP MMAs are complete, and its first
 // MMAs run while the current item's dQ is still being stored.
-// PACKED: the index holds document bounds.  The kernel proper picks one of the two bodies by the
-// index header's `packed` word; without the bounds every test for them is compiled out (as
+// PACKED: the index holds document bounds.  There is one kernel per body (see bwd_dq_kernel);
+// without the bounds every test for them is compiled out (as
 // run-time tests they cost this kernel, which decodes an item in every role, 8 % of its time).
 template <int D, bool PACKED>
 __device__ __forceinline__ void
@@ -442,14 +442,18 @@ bwd_dq_body(const CUtensorMap& mapK, const CUtensorMap& mapV, const CUtensorMap&
   if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int D>
+// Both instances are launched, one after the other; the one that does not match the index
+// header's `packed` word returns at once (the host cannot read that word without a
+// synchronisation).  One kernel holding both bodies ran the common one 3 % slower than it runs
+// alone, and a called (not inlined) second body 17 % slower; an empty launch costs 2-3 us.
+template <int D, bool PACKED>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
               const __grid_constant__ CUtensorMap mapKs, const __grid_constant__ CUtensorMap mapVs,
               const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ dOg,
               const BwdParams p, const int n_items) {
-  if (p.index_header->packed) bwd_dq_body<D, true>(mapK, mapV, mapKs, mapVs, Qg, dOg, p, n_items);
-  else bwd_dq_body<D, false>(mapK, mapV, mapKs, mapVs, Qg, dOg, p, n_items);
+  if ((p.index_header->packed != 0) != PACKED) return;
+  bwd_dq_body<D, PACKED>(mapK, mapV, mapKs, mapVs, Qg, dOg, p, n_items);
 }
 
 // ---------------------------------------------------------------------------
@@ -957,7 +961,11 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   p.scale = (d->scale != 0.f) ? d->scale : 1.0f / sqrtf(float(d->d));
   p.scale_log2 = p.scale * kLog2e;
 
-  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dq_kernel<D, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       int(DqCfg<D>::kRequest)));
+  SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dq_kernel<D, true>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        int(DqCfg<D>::kRequest)));
   SEPLLM_CUDA_TRY(cudaFuncSetAttribute(bwd_dkv_kernel<D, true>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -967,7 +975,10 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
                                        int(DkvCfg<D>::kRequest)));
   {
     const int n_items = d->Hq * d->B * ih.n_tiles;
-    bwd_dq_kernel<D><<<std::min(n_items, sm_count()), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
+    bwd_dq_kernel<D, false><<<std::min(n_items, sm_count()), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
+        mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO),
+        p, n_items);
+    bwd_dq_kernel<D, true><<<std::min(n_items, sm_count()), kBwdThreads, DqCfg<D>::kRequest, stream>>>(
         mk, mv, mks, mvs, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO),
         p, n_items);
   }

@@ -165,9 +165,9 @@ class Workload:
         self.dV = torch.empty_like(self.V)
         self.out_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (self.O, self.dQ, self.dK, self.dV)]
         # index scan | side gather, forward | Delta, dQ, dK/dV side, dK/dV window
-        # index; gather + forward; delta + dQ (two instances, the one that does not match the index
+        # index (clear + scan); gather + forward; delta + dQ (two instances, the one that does not match the index
         # returns at once) + dK/dV side + dK/dV window
-        self.launches_per_step = 1 + 2 + (0 if fwd_only else 5)
+        self.launches_per_step = 2 + 2 + (0 if fwd_only else 5)
 
     def step(self, bufs=None):
         api = self.api

@@ -904,7 +904,7 @@ static sepllm_status launch_bwd(const sepllm_attn_desc* d, const sepllm_index_de
   const int32_t* n_side = reinterpret_cast<const int32_t*>(index + ih.off_n_side);
   record_event(d, 0, stream);
   if (!(d->flags & SEPLLM_ATTN_SIDE_READY))
-    launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
+    launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, reinterpret_cast<int32_t*>(ws), stream);
   record_event(d, 1, stream);
 
   float2* stats = reinterpret_cast<float2*>(ws + lay.off_delta);
@@ -1017,7 +1017,7 @@ extern "C" sepllm_status sepllm_attn_bwd(const sepllm_attn_desc* desc,
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   // A backward that continues on the forward's workspace keeps the forward's status word: a
   // condition the forward recorded stays readable until the caller looks at it.
-  if (!(desc->flags & SEPLLM_ATTN_SIDE_READY)) SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
+  // Otherwise the side gather, the call's first launch, resets it.
   const uint8_t* idx = static_cast<const uint8_t*>(index);
   if (kernel_head_dim(desc->d) == 64)
     return launch_bwd<64>(desc, idesc, ih, dO, Q, K, V, O, LSE, idx, dQ, dK, dV, ws, stream);

@@ -149,7 +149,7 @@ __global__ void gather_side_kv(const __nv_bfloat16* __restrict__ K,
                                const int32_t* __restrict__ side_pos,
                                const int32_t* __restrict__ n_side, int L, int d, int Hkv,
                                int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
-                               __nv_bfloat16* __restrict__ Vs);
+                               __nv_bfloat16* __restrict__ Vs, int32_t* __restrict__ status);
 
 // Forward for groups of four query heads at head size 128: two CTAs of a cluster work on the four
 // heads of one query tile as one MMA pair (attn_fwd_pair.cu).  Ks64 / K64: maps with 64-row boxes.
@@ -173,8 +173,10 @@ inline void record_event(const sepllm_attn_desc* d, int i, cudaStream_t stream) 
 }
 
 // Launches the gather of K/V rows at the side positions into Ks / Vs ([B][Hkv][cap_pad][D]).
+// The gather is the first launch of a call that runs it, and it resets the workspace's status word
+// (one thread) instead of a memset node in front of it.
 void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
                    const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
-                   void* Ks, void* Vs, cudaStream_t stream);
+                   void* Ks, void* Vs, int32_t* status, cudaStream_t stream);
 
 }  // namespace sepllm

@@ -58,10 +58,11 @@ __global__ void __launch_bounds__(256)
 gather_side_kv(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                const int32_t* __restrict__ side_pos, const int32_t* __restrict__ n_side, int L,
                int d, int Hkv, int side_cap, int cap_pad, __nv_bfloat16* __restrict__ Ks,
-               __nv_bfloat16* __restrict__ Vs) {
+               __nv_bfloat16* __restrict__ Vs, int32_t* __restrict__ status) {
   constexpr int LPR = D / 8;
   constexpr int RPB = 256 / LPR;
   const int b = blockIdx.z, hk = blockIdx.y;
+  if (threadIdx.x == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) *status = SEPLLM_OK;
   const int r = blockIdx.x * RPB + threadIdx.x / LPR, l = threadIdx.x % LPR;
   const int ns = min(n_side[b], side_cap);
   const int ns_pad = min(cap_pad, (ns + 127) / 128 * 128);
@@ -470,19 +471,19 @@ AttnLayout attn_layout(const sepllm_attn_desc* d, const sepllm_index_desc* id) {
 
 void launch_gather(const sepllm_attn_desc* d, const sepllm_index_desc* id, int cap_pad,
                    const void* K, const void* V, const int32_t* side_pos, const int32_t* n_side,
-                   void* Ks, void* Vs, cudaStream_t stream) {
+                   void* Ks, void* Vs, int32_t* status, cudaStream_t stream) {
   if (kernel_head_dim(d->d) == 64) {
     constexpr int RPB = 256 / (64 / 8);
     gather_side_kv<64><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
         n_side, d->L, d->d, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
-        static_cast<__nv_bfloat16*>(Vs));
+        static_cast<__nv_bfloat16*>(Vs), status);
   } else {
     constexpr int RPB = 256 / (128 / 8);
     gather_side_kv<128><<<dim3((cap_pad + RPB - 1) / RPB, d->Hkv, d->B), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), side_pos,
         n_side, d->L, d->d, d->Hkv, id->side_cap, cap_pad, static_cast<__nv_bfloat16*>(Ks),
-        static_cast<__nv_bfloat16*>(Vs));
+        static_cast<__nv_bfloat16*>(Vs), status);
   }
 }
 
@@ -498,7 +499,7 @@ static sepllm_status launch_fwd(const sepllm_attn_desc* d, const sepllm_index_de
   const int32_t* n_side = reinterpret_cast<const int32_t*>(index + ih.off_n_side);
   record_event(d, 0, stream);
   if (!(d->flags & SEPLLM_ATTN_SIDE_READY))
-    launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, stream);
+    launch_gather(d, id, lay.cap_pad, K, V, side_pos, n_side, Ks, Vs, reinterpret_cast<int32_t*>(ws), stream);
   record_event(d, 1, stream);
 
   CUtensorMap mq, mk, mv, mks, mvs;
@@ -574,7 +575,8 @@ extern "C" sepllm_status sepllm_attn_fwd(const sepllm_attn_desc* desc,
   if ((st = fill_index_header(idesc, &ih)) != SEPLLM_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, kAlign, stream));
+  // (the side gather, the call's first launch, resets the status word)
+  if (desc->flags & SEPLLM_ATTN_SIDE_READY) SEPLLM_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(int32_t), stream));
   if (kernel_head_dim(desc->d) == 64)
     return launch_fwd<64>(desc, idesc, ih, Q, K, V, static_cast<const uint8_t*>(index), O, LSE, ws,
                           stream);

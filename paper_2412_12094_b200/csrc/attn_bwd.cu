@@ -339,6 +339,17 @@ bwd_dq_body(const CUtensorMap& mapK, const CUtensorMap& mapV, const CUtensorMap&
     for (; w < n_items; ++ino) {
       const DqItem it = dq_item(p, dv, w);
       const int w_next = next_item(w + gridDim.x);
+      // The next item's Q / dO row is loaded at the hand-over between items, where the tensor pipe
+      // waits for it: ask for its lines now, a whole item ahead, so that the load finds them in L2.
+      if (w_next < n_items) {
+        const DqItem nx = dq_item(p, dv, w_next);
+        const int nrow = nx.t * kBM + r;
+        if (nrow < p.L) {
+          const char* a = reinterpret_cast<const char*>((u ? dOg : Qg) + (size_t(nx.q_plane) * p.L + nrow) * p.d);
+          for (int off = 0; off < p.d * 2; off += 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(a + off));
+        }
+      }
       const int t = it.t, ns = it.ns;
       const int row = t * kBM + r;
       const bool row_ok = row < p.L;

@@ -193,7 +193,7 @@ sepllm_status sepllm_build_index_varlen(const sepllm_index_desc* desc, const int
  * attention calls read the header's `packed` word on the device and follow
  * the document bounds; sepllm_cache_from_prompt takes no such index.
  * scratch is not used (may be NULL).  Integer output, deterministic; a plain
- * multi-pass build (one block per row scans it in 1024-token steps), not
+ * multi-pass build (one block per row scans it in 8192-token steps), not
  * tuned like sepllm_build_index. */
 sepllm_status sepllm_build_index_packed(const sepllm_index_desc* desc, const int32_t* token_ids,
                                         const int32_t* doc_first, const int32_t* seq_len,

@@ -1,7 +1,7 @@
 // Index of rows that pack several documents: sepllm_build_index_packed.
 //
 // Three plain passes (this variant is not on the timed path):
-//   packed_scan   one block per row walks it in 1024-token steps, forwards for the document
+//   packed_scan   one block per row walks it in 8192-token steps, forwards for the document
 //                 starts (running maximum of the boundary positions), the side members and their
 //                 prefix counts, then backwards for the document ends (running minimum);
 //   packed_rows   lim[i] = cnt[max(i-n+1, doc_start[i])] for every position;
@@ -12,22 +12,37 @@ namespace sepllm {
 
 constexpr int kScanThreads = 1024;
 
-// Inclusive scan over the block's 1024 values in shared memory (log-step, two barriers a step).
-// REVERSE scans from the last thread towards the first.
+// Scan over the block's 1024 values, in thread order or (REVERSE) from the last thread towards the
+// first: warp shuffles, then the warps' totals through shared memory (sh: 32 words; two barriers a
+// call).  incl includes the thread's own value, excl does not (identity for the first in order).
+struct ScanResult {
+  int incl, excl;
+};
 template <bool REVERSE, class Op>
-__device__ __forceinline__ int block_scan(int v, int* sh, Op op) {
-  const int tid = REVERSE ? kScanThreads - 1 - int(threadIdx.x) : int(threadIdx.x);
-  sh[tid] = v;
-  __syncthreads();
-  for (int o = 1; o < kScanThreads; o <<= 1) {
-    const int other = (tid >= o) ? sh[tid - o] : v;
-    __syncthreads();
-    if (tid >= o) v = op(v, other);
-    sh[tid] = v;
-    __syncthreads();
+__device__ __forceinline__ ScanResult block_scan(int v, int* sh, Op op, int identity) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = REVERSE ? __shfl_down_sync(0xffffffffu, x, o) : __shfl_up_sync(0xffffffffu, x, o);
+    if (REVERSE ? (lane + o < 32) : (lane >= o)) x = op(x, y);
   }
-  return v;
+  if (lane == (REVERSE ? 0 : 31)) sh[w] = x;
+  __syncthreads();
+  int acc = identity;   // everything in the warps before this one in scan order
+  if (REVERSE) { for (int k = kScanThreads / 32 - 1; k > w; --k) acc = op(acc, sh[k]); }
+  else { for (int k = 0; k < w; ++k) acc = op(acc, sh[k]); }
+  __syncthreads();
+  const int nb = REVERSE ? __shfl_down_sync(0xffffffffu, x, 1) : __shfl_up_sync(0xffffffffu, x, 1);
+  const bool first_in_warp = REVERSE ? (lane == 31) : (lane == 0);
+  ScanResult r;
+  r.incl = op(acc, x);
+  r.excl = first_in_warp ? acc : op(acc, nb);
+  return r;
 }
+
+constexpr int kScanItems = 8;                          // consecutive positions per thread
+constexpr int kScanStep = kScanThreads * kScanItems;   // positions per step of the walk
 
 __global__ void __launch_bounds__(kScanThreads)
 packed_scan(const int32_t* __restrict__ token_ids, const int32_t* __restrict__ doc_first,
@@ -35,7 +50,7 @@ packed_scan(const int32_t* __restrict__ token_ids, const int32_t* __restrict__ d
             int32_t* __restrict__ cnt, int32_t* __restrict__ side_pos, int32_t* __restrict__ n_side,
             int32_t* __restrict__ doc_start, int32_t* __restrict__ doc_end,
             int32_t* __restrict__ seq_len_out, int32_t* status) {
-  __shared__ int sh[kScanThreads];
+  __shared__ int sh[kScanThreads / 32];
   __shared__ int carry_a, carry_b;
   const int b = blockIdx.x, tid = threadIdx.x;
   const int Lv = seq_len ? max(0, min(L, seq_len[b])) : L;
@@ -50,28 +65,49 @@ packed_scan(const int32_t* __restrict__ token_ids, const int32_t* __restrict__ d
   auto iadd = [](int x, int y) { return x + y; };
   if (tid == 0) { carry_a = 0; carry_b = 0; }   // document start so far, members so far
   __syncthreads();
-  for (int base = 0; base < L; base += kScanThreads) {
-    const int j = base + tid;
-    const bool valid = j < Lv;
-    const bool bnd = valid && (j == 0 || df[j] != 0);
+  // ---- forwards: document starts, members, prefix counts ----
+  for (int base = 0; base < L; base += kScanStep) {
+    const int j0 = base + tid * kScanItems;
     const int start_before = carry_a, members_before = carry_b;
     // boundaries only grow along the row, so their running maximum is the nearest one so far
-    const int scan = block_scan<false>(bnd ? j : -1, sh, imax);
-    const int start = valid ? max(scan, start_before) : j;   // padding belongs to no document
-    const bool member = valid && (j - start < n_init || is_separator(ids[j], sep));
-    const int incl = block_scan<false>(member ? 1 : 0, sh, iadd);
-    const int c = members_before + incl - (member ? 1 : 0);
-    if (j < L) {
-      cnt_b[j] = c;
-      ds[j] = start;
-      if (member) {
-        if (c < side_cap) sp[c] = j;
-        else set_status(status, SEPLLM_CAPACITY_EXCEEDED);
+    int start[kScanItems], tok[kScanItems];
+    int run = -1;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      const int j = j0 + k;
+      const bool valid = j < Lv;
+      tok[k] = valid ? ids[j] : 0;
+      if (valid && (j == 0 || df[j] != 0)) run = j;
+      start[k] = run;
+    }
+    const int before = max(block_scan<false>(run, sh, imax, -1).excl, start_before);
+    uint32_t member = 0;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      const int j = j0 + k;
+      const bool valid = j < Lv;
+      start[k] = valid ? max(start[k], before) : j;   // padding belongs to no document
+      if (valid && (j - start[k] < n_init || is_separator(tok[k], sep))) member |= 1u << k;
+    }
+    const int n_mine = __popc(member);
+    const ScanResult ms = block_scan<false>(n_mine, sh, iadd, 0);
+    int c = members_before + ms.excl;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      const int j = j0 + k;
+      if (j < L) {
+        cnt_b[j] = c;
+        ds[j] = start[k];
+        if ((member >> k) & 1u) {
+          if (c < side_cap) sp[c] = j;
+          else set_status(status, SEPLLM_CAPACITY_EXCEEDED);
+          ++c;
+        }
       }
     }
     if (tid == kScanThreads - 1) {   // (every thread read the carries before the scans' barriers)
-      carry_a = max(scan, start_before);
-      carry_b = members_before + incl;
+      carry_a = max(max(run, before), start_before);
+      carry_b = members_before + ms.incl;
     }
     __syncthreads();
   }
@@ -82,22 +118,31 @@ packed_scan(const int32_t* __restrict__ token_ids, const int32_t* __restrict__ d
     seq_len_out[b] = Lv;
   }
   for (int r = total + tid; r < side_cap; r += kScanThreads) sp[r] = -1;
-  // document ends: the nearest boundary after j, else the end of the row's tokens
+  // ---- backwards: document ends = the nearest boundary after j, else the end of the row's tokens ----
   __syncthreads();
   if (tid == 0) carry_a = Lv;
   __syncthreads();
-  const int n_steps = (L + kScanThreads - 1) / kScanThreads;
+  const int n_steps = (L + kScanStep - 1) / kScanStep;
   for (int step = n_steps - 1; step >= 0; --step) {
-    const int j = step * kScanThreads + tid;
-    const bool valid = j < Lv;
-    const bool bnd = valid && (j == 0 || df[j] != 0);
+    const int j0 = step * kScanStep + tid * kScanItems;
     const int end_after = carry_a;
-    const int incl = block_scan<true>(bnd ? j : 0x7fffffff, sh, imin);   // boundaries at or after j in the step
-    // block_scan<true> leaves thread t's result at sh[1023 - t]: thread tid + 1's sits at sh[1022 - tid]
-    const int after = (tid + 1 < kScanThreads) ? sh[kScanThreads - 2 - tid] : 0x7fffffff;
-    if (j < L) de[j] = valid ? min(after, end_after) : j;
+    int nxt[kScanItems];   // nearest boundary after position k among this thread's own positions
+    int run = 0x7fffffff;
+#pragma unroll
+    for (int k = kScanItems - 1; k >= 0; --k) {
+      const int j = j0 + k;
+      nxt[k] = run;
+      if (j < Lv && (j == 0 || df[j] != 0)) run = j;
+    }
+    const ScanResult sr = block_scan<true>(run, sh, imin, 0x7fffffff);
+    const int after = min(sr.excl, end_after);   // boundaries in later threads and later steps
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      const int j = j0 + k;
+      if (j < L) de[j] = (j < Lv) ? min(nxt[k], after) : j;
+    }
     __syncthreads();
-    if (tid == 0) carry_a = min(incl, end_after);
+    if (tid == 0) carry_a = min(sr.incl, end_after);
     __syncthreads();
   }
 }
